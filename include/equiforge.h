@@ -1,0 +1,139 @@
+/*
+ * equiforge.h -- C ABI of the B200 (sm_100a) fused tensor-program library.
+ *
+ * One entry point per fused program that the paper's equality-saturation
+ * superoptimizer rewrites and extracts (Section 7.1 "Workloads": normalisation,
+ * MLPs, low-rank adaptation, multi-head attention in decode and prefill).  The
+ * library executes those programs; the e-graph search is not part of it.
+ *
+ * Conventions common to every entry point
+ *   - All tensor pointers are DEVICE pointers to bfloat16 data (1-8-7 format),
+ *     row-major, contiguous, last dimension fastest, 16-byte aligned.
+ *     Arithmetic is bf16 x bf16 -> fp32 accumulate (Figure 4: "acc=f32"); outputs are
+ *     rounded to bf16 with round-to-nearest-even.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *     Calls are asynchronous: they enqueue 1..3 kernels and return without synchronising.
+ *   - `ws` is a caller-owned DEVICE scratch buffer of at least
+ *     ef_<program>_workspace_bytes(...) bytes, 256-byte aligned.  It must be initialised
+ *     ONCE with ef_workspace_init() (or zero-filled) before its first use; afterwards the
+ *     library keeps its bookkeeping words consistent across calls.  One workspace serves one
+ *     call at a time: two calls that may overlap on the GPU need two workspaces.  Apart
+ *     from the first 256 bytes (status + bookkeeping) its contents are undefined after a call.
+ *   - Ownership: the caller owns every buffer and the stream.  The library allocates no
+ *     device memory, frees nothing, and keeps only host-side caches (driver entry point,
+ *     kernel attributes, SM count).  Inputs are read-only; the output is fully overwritten.
+ *     An output that aliases an input is undefined behaviour.
+ *   - Errors: return codes only (no exceptions, no abort, no device trap).  Argument errors
+ *     are detected on the host before anything is enqueued.  Every device-side wait is
+ *     bounded; a wait that gives up records EF_ERR_DEVICE_TIMEOUT in the workspace status
+ *     word, the kernel drains and exits normally, and ef_check_status() reports it.
+ *   - There is no CPU fallback: a shape outside the supported set returns
+ *     EF_ERR_UNSUPPORTED, a device that is not compute capability 10.x returns EF_ERR_ARCH.
+ */
+#ifndef EQUIFORGE_H_
+#define EQUIFORGE_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EF_OK = 0,
+    EF_ERR_NULL = 1,           /* a required pointer is NULL                                   */
+    EF_ERR_SHAPE = 2,          /* non-positive or inconsistent dimensions                      */
+    EF_ERR_UNSUPPORTED = 3,    /* valid problem, but no kernel covers it (see each entry)      */
+    EF_ERR_ALIGN = 4,          /* pointer not 16-byte aligned (workspace: 256-byte)            */
+    EF_ERR_WORKSPACE = 5,      /* ws == NULL or ws_bytes below the query                       */
+    EF_ERR_ARCH = 6,           /* current device is not compute capability 10.x                */
+    EF_ERR_CUDA = 7,           /* a CUDA runtime/driver call failed; see ef_last_cuda_error()  */
+    EF_ERR_DEVICE_TIMEOUT = 8  /* a bounded device-side wait gave up (ef_check_status only)    */
+} ef_status;
+
+/* ---- Program 1: fused RMSNorm + matmul ---------------------------------------------------
+ * Y = (X * rsqrt(mean(X^2, -1) + eps) * gamma) @ W.
+ * Definition: RMSNorm expanded into reduce + pointwise ops feeding a MatMul (Section 7.1,
+ * "Implementation"); the per-row factor is invariant along K and is applied after the
+ * contraction (Table 1, factor motion; Section 7.2, RMSNorm-MLP discussion), gamma stays on
+ * the X side; the sum of squares and the K loop form one fused reduction (Table 1, product
+ * fusion); W is partitioned along N and K (Table 1, MatMul refinement "NK").
+ *   X [M,K], gamma [K], W [K,N] -> Y [M,N].
+ * Supported: 1 <= M <= 16, K % 64 == 0, N % 8 == 0. */
+ef_status ef_rmsnorm_matmul(const void* X, const void* gamma, const void* W, void* Y,
+                            int M, int K, int N, float eps,
+                            void* ws, size_t ws_bytes, void* stream);
+size_t ef_rmsnorm_matmul_workspace_bytes(int M, int K, int N);
+
+/* ---- Program 2: fused gated MLP (SwiGLU) -------------------------------------------------
+ * Y = SiLU(X @ Wgate) * (X @ Wup), SiLU(z) = z / (1 + exp(-z)).
+ * Definition: the GatedMLP workload of Section 7.1 / Table 2; both projections and the
+ * elementwise product run in one kernel (Section 7.2).  K-partitioned partial products are
+ * summed (Reduce over the parallel K axis, Table 1 "NK") BEFORE the nonlinear gate.
+ *   X [M,K], Wgate [K,N], Wup [K,N] -> Y [M,N].
+ * Supported: 1 <= M <= 16, K % 64 == 0, N % 8 == 0. */
+ef_status ef_gated_mlp(const void* X, const void* Wgate, const void* Wup, void* Y,
+                       int M, int K, int N,
+                       void* ws, size_t ws_bytes, void* stream);
+size_t ef_gated_mlp_workspace_bytes(int M, int K, int N);
+
+/* ---- Program 3: grouped-query decode attention -------------------------------------------
+ * One query token per sequence attends all L cached keys: for query head h and kv head
+ * g = h / (Hq/Hkv):  O[b,h] = softmax_j(scale * Q[b,h] . K[b,g,j]) @ V[b,g].
+ * Definition: vanilla attention M0 of Figure 4, executed as the tiled rolling form M2
+ * (state <max,sum,value>, repair h(c,s,s') = c*exp(s-s'), Section 4.2); the key axis is also
+ * split across thread blocks and the partial states are stored and merged (Table 1,
+ * intermediate storage; Section 4.4).
+ *   Q [B,Hq,D], K [B,Hkv,L,D], V [B,Hkv,L,D] -> O [B,Hq,D].
+ * Supported: D == 128, Hq % Hkv == 0, Hq/Hkv <= 16, L >= 1. */
+ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O,
+                        int B, int Hq, int Hkv, int L, int D, float scale,
+                        void* ws, size_t ws_bytes, void* stream);
+size_t ef_gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int L, int D);
+
+/* ---- Program 4: QK-normalised (causal) prefill attention ---------------------------------
+ * qh = q * rsqrt(mean_d q^2 + eps) * gamma_q, kh likewise with gamma_k (over head_dim);
+ * s_ij = scale * qh_i . kh_j for j <= i when causal != 0 (all j otherwise); softmax over j;
+ * O = P @ V.  Definition: M0 -> M2 of Figure 4 with RMSNorm on Q and K; the inverse-RMS
+ * factors are invariant along the contraction and move onto the logits (Table 1, factor
+ * motion; Section 7.3, QK-normalized MLA).  Score and probability matrices never reach HBM
+ * (Section 7.2, "Attention").
+ *   Q,K,V [B,H,S,D], gamma_q [D], gamma_k [D] -> O [B,H,S,D].
+ * Supported: D == 128, S >= 1. */
+ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V,
+                         const void* gamma_q, const void* gamma_k, void* O,
+                         int B, int H, int S, int D, float eps, float scale, int causal,
+                         void* ws, size_t ws_bytes, void* stream);
+size_t ef_qknorm_attn_workspace_bytes(int B, int H, int S, int D);
+
+/* ---- Program 5: LoRA-fused linear ---------------------------------------------------------
+ * Y = X @ W + alpha * (X @ A) @ Bm.
+ * Definition: the LoRA workload (Section 7.1; Figure 2 factoring; Table 1 MatMul
+ * reassociation).  Executed in the two-kernel form the paper's search selects (Section 7.2):
+ * T = alpha * (X @ A) is stored once, then Y = [X | T] @ [W ; Bm] adds the rank-R update as
+ * one extra K slab of the main contraction.
+ *   X [M,K], W [K,N], A [K,R], Bm [R,N] -> Y [M,N].
+ * Supported: R == 16, K % 64 == 0, N % 8 == 0. */
+ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void* Bm, void* Y,
+                         int M, int K, int N, int R, float alpha,
+                         void* ws, size_t ws_bytes, void* stream);
+size_t ef_lora_linear_workspace_bytes(int M, int K, int N, int R);
+
+/* ---- Workspace and status -------------------------------------------------------------------
+ * (No counterpart in the paper: library plumbing.)
+ * ef_workspace_init: enqueue zero-fill of the first min(ws_bytes, 64 KiB) bytes of ws on
+ *   `stream` (status word, cross-block arrival counters).  Call once per workspace, and again
+ *   after ef_check_status reported EF_ERR_DEVICE_TIMEOUT.
+ * ef_check_status: synchronise `stream`, read the 4-byte status word at ws[0]; returns EF_OK,
+ *   EF_ERR_DEVICE_TIMEOUT, or EF_ERR_CUDA if the stream itself failed. */
+ef_status ef_workspace_init(void* ws, size_t ws_bytes, void* stream);
+ef_status ef_check_status(const void* ws, void* stream);
+
+const char* ef_status_string(ef_status s);
+int ef_last_cuda_error(void); /* last cudaError_t / CUresult seen by this thread's failing call */
+int ef_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EQUIFORGE_H_ */

@@ -1,0 +1,44 @@
+// Host-side plumbing shared by the entry points: argument checks, the cached driver entry
+// point for tensor-map encoding, device properties, error bookkeeping.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/equiforge.h"
+
+namespace ef {
+
+// Workspace header: [0,16) status word, [16,256) reserved, [256, kHeaderBytes) arrival counters.
+constexpr size_t kHeaderBytes = 4096;
+constexpr size_t kCounterOffset = 256;
+constexpr size_t kMaxCounters = (kHeaderBytes - kCounterOffset) / sizeof(uint32_t);  // 960
+
+extern thread_local int g_last_cuda_error;
+
+struct DeviceInfo {
+    int device = -1;
+    int cc_major = 0;
+    int num_sms = 0;
+    int max_smem_optin = 0;
+};
+// Properties of the CURRENT device (cached per device id).  Returns false on CUDA failure.
+bool current_device_info(DeviceInfo* out);
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Encode a tiled tensor map over bf16 data.  dims/box are innermost-first; strides_bytes[i] is
+// the byte stride of dimension i+1 (rank-1 entries).  swizzle: CU_TENSOR_MAP_SWIZZLE_*.
+ef_status encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+                           const uint64_t* strides_bytes, const uint32_t* box, CUtensorMapSwizzle swizzle);
+
+#define EF_CUDA_CHECK(expr)                                  \
+    do {                                                     \
+        cudaError_t _e = (expr);                             \
+        if (_e != cudaSuccess) {                             \
+            ::ef::g_last_cuda_error = static_cast<int>(_e);  \
+            return EF_ERR_CUDA;                              \
+        }                                                    \
+    } while (0)
+
+}  // namespace ef

@@ -85,7 +85,7 @@ size_t ef_gated_mlp_workspace_bytes(int M, int K, int N);
  * split across thread blocks and the partial states are stored and merged (Table 1,
  * intermediate storage; Section 4.4).
  *   Q [B,Hq,D], K [B,Hkv,L,D], V [B,Hkv,L,D] -> O [B,Hq,D].
- * Supported: D == 128, Hq % Hkv == 0, Hq/Hkv <= 16, L >= 1. */
+ * Supported: D == 128, Hq % Hkv == 0, Hq/Hkv <= 8, L >= 1. */
 ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O,
                         int B, int Hq, int Hkv, int L, int D, float scale,
                         void* ws, size_t ws_bytes, void* stream);

@@ -6,13 +6,16 @@
 // traversed by a loop that carries the rolling state <max, sum, value> (the parallel reduce axis
 // becomes an in-block loop, Section 6.1); where a unit's chunks are spread over several blocks the
 // partial states are stored (Collection) and merged by the block that arrives last, using the same
-// associative reducer, in a fixed order (deterministic, no floating-point atomics).
+// associative reducer, in block order (deterministic, no floating-point atomics).
 //
-// Data movement: a producer warp streams K and V chunks with TMA (128-byte swizzle) through a
-// 3-stage, 64 KiB-per-stage shared-memory ring, so ~192 KiB per SM are in flight.  Four consumer
-// warps each own 32 keys of every chunk: QK^T and PV run on warp-level mma.sync (the 4..16 query
-// heads that share a kv head are the M rows of the MMA), softmax statistics are reduced with
-// warp shuffles.  The kernel moves 2 bytes per 4 flops; tcgen05 would not help it.
+// Data movement: a producer thread streams K and V chunks with TMA (128-byte swizzle) through a
+// 3-stage, 64 KiB-per-stage shared-memory ring, so ~192 KiB per SM are in flight (a plain
+// streaming kernel with this ring reads 128 MiB in ~25 us on a B200; stages of 16 KiB or less lose
+// 15-40 % of that).  Four consumer warps each own 32 keys of every chunk: QK^T and PV run on
+// warp-level mma.sync (the <= 8 query heads that share a kv head are the M rows of the MMA),
+// softmax statistics are reduced with warp shuffles.  The kernel moves 2 bytes per 4 flops;
+// tcgen05 would not help it.  All index arithmetic on the merge path is 32-bit: a 64-bit division
+// per element there once cost more than the whole data stream.
 #include "host.cuh"
 #include "ptx.cuh"
 
@@ -28,11 +31,12 @@ constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;
 constexpr int kKeysPerWarp = kChunk / kConsumerWarps;  // 32
-constexpr int kMaxGroup = 16;                     // query heads per kv head (rows of the MMA)
-constexpr int kRowFloats = kD + 2;                // m, l, value[128]
+constexpr int kMaxGroup = 8;                      // query heads per kv head (rows 0..7 of the MMA)
+constexpr int kRowFloats = kD + 4;                // value[128], m, l, 2 pad (rows stay 16-byte aligned)
 constexpr int kSlotFloats = kMaxGroup * kRowFloats;
 constexpr int kMergeBytes = kConsumerWarps * kSlotFloats * 4;
-constexpr int kBarBytes = 128;
+constexpr int kMaxGrid = 256;                     // upper bound on the persistent grid
+constexpr int kBarBytes = 128 + kMaxGrid * 4;     // barriers, flags, slot table of the final merge
 constexpr int kSmemBytes = 1024 /*align slack*/ + kStages * kStageBytes + kMergeBytes + kBarBytes;
 
 struct Params {
@@ -40,7 +44,8 @@ struct Params {
     __nv_bfloat16* O;
     int B, Hq, Hkv, L, G;
     int n_chunks;      // chunks per (b, kv head) unit
-    int total_items;   // units * n_chunks
+    int total_items;   // units * n_chunks  (< 2^30)
+    int base, rem;     // block c owns base + (c < rem) consecutive items
     float scale_log2;  // scale * log2(e)
     uint32_t* status;
     uint32_t* counters;  // one arrival counter per unit, zero between calls
@@ -52,16 +57,18 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
                                           uint32_t* status, uint32_t site) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, site)) != 0;
 }
-
-__device__ __forceinline__ long long range_begin(int cta, int n_cta, int total) {
-    return (static_cast<long long>(cta) * total) / n_cta;
+__device__ __forceinline__ void consumer_sync() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
 }
-// Block that owns item x under the contiguous partition range_begin().
-__device__ __forceinline__ int owner_of(long long x, int n_cta, int total) {
-    int c = static_cast<int>(((x + 1) * n_cta - 1) / total);
-    while (c > 0 && range_begin(c, n_cta, total) > x) --c;
-    while (c + 1 < n_cta && range_begin(c + 1, n_cta, total) <= x) ++c;
-    return c;
+// Contiguous partition of the item list (32-bit arithmetic only).
+__device__ __forceinline__ int range_begin(int c, int base, int rem) { return c * base + min(c, rem); }
+__device__ __forceinline__ int owner_of(int x, int base, int rem) {
+    const int big = rem * (base + 1);
+    return x < big ? x / (base + 1) : rem + (x - big) / base;
+}
+// Partial-state slot of block c for `unit`: 0 if the unit is the first one the block touches, else 1.
+__device__ __forceinline__ int slot_of(int c, int unit, int base, int rem, int n_chunks) {
+    return 2 * c + ((range_begin(c, base, rem) / n_chunks) == unit ? 0 : 1);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -76,13 +83,13 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     uint64_t* empty = bars + 2 * kStages;   // [kStages]
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 3 * kStages);
     uint32_t* is_last = const_cast<uint32_t*>(abort_flag) + 1;
+    int* slot_table = reinterpret_cast<int*>(bars) + 32;  // [kMaxGrid]
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-    const int n_cta = gridDim.x;
-    const long long it_begin = range_begin(blockIdx.x, n_cta, p.total_items);
-    const long long it_end = range_begin(blockIdx.x + 1, n_cta, p.total_items);
+    const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
+    const int it_end = range_begin(blockIdx.x + 1, p.base, p.rem);
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -103,11 +110,12 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             tma_prefetch_desc(&tmV);
             int stage = 0;
             uint32_t phase = 0;
-            for (long long it = it_begin; it < it_end; ++it) {
-                const int unit = static_cast<int>(it / p.n_chunks);
-                const int key0 = static_cast<int>(it % p.n_chunks) * kChunk;
+            int unit = it_begin / p.n_chunks;
+            int chunk = it_begin - unit * p.n_chunks;
+            for (int it = it_begin; it < it_end; ++it) {
                 if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) break;
                 uint8_t* st = stages + stage * kStageBytes;
+                const int key0 = chunk * kChunk;
                 mbar_expect_tx(&fullK[stage], 2 * kHalfBytes);
                 tma_load_3d(st, &tmK, &fullK[stage], 0, key0, unit);
                 tma_load_3d(st + kHalfBytes, &tmK, &fullK[stage], 64, key0, unit);
@@ -115,43 +123,42 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 tma_load_3d(st + 2 * kHalfBytes, &tmV, &fullV[stage], 0, key0, unit);
                 tma_load_3d(st + 3 * kHalfBytes, &tmV, &fullV[stage], 64, key0, unit);
                 if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                if (++chunk == p.n_chunks) { chunk = 0; ++unit; }
             }
         }
     } else {
         // ------------------------------ consumer warps -----------------------------
-        const int g = lane >> 2;        // fragment row (query head within the group), also row g+8
+        const int g = lane >> 2;        // fragment row = query head within the group (rows 8..15 are padding)
         const int t4 = lane & 3;
         int stage = 0;
         uint32_t phase = 0;
-        long long it = it_begin;
+        int it = it_begin;
         bool ok = true;
         while (it < it_end && ok) {
-            const int unit = static_cast<int>(it / p.n_chunks);
-            const int c0 = static_cast<int>(it % p.n_chunks);
-            const long long unit_end = static_cast<long long>(unit + 1) * p.n_chunks;
-            const long long seg_end = unit_end < it_end ? unit_end : it_end;
-            const int n_seg = static_cast<int>(seg_end - it);
+            const int unit = it / p.n_chunks;
+            const int c0 = it - unit * p.n_chunks;
+            const int unit_end = (unit + 1) * p.n_chunks;
+            const int seg_end = unit_end < it_end ? unit_end : it_end;
+            const int n_seg = seg_end - it;
             const bool whole_unit = (c0 == 0) && (seg_end == unit_end);
-            const int b = unit / p.Hkv, kvh = unit % p.Hkv;
+            const int b = unit / p.Hkv, kvh = unit - b * p.Hkv;
             const int head0 = kvh * p.G;
 
             // Q fragments (A operand, 16 x 128): rows >= G are zero padding.
             uint32_t qf[8][4];
             {
                 const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.Q + (static_cast<size_t>(b) * p.Hq + head0 + g) * kD);
-                const uint32_t* q1 = q0 + 8 * (kD / 2);
-                const bool r0 = g < p.G, r1 = (g + 8) < p.G;
+                const bool r0 = g < p.G;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const int c = ks * 8 + t4;  // uint32 index of column ks*16 + 2*t4
                     qf[ks][0] = r0 ? __ldg(q0 + c) : 0u;
-                    qf[ks][1] = r1 ? __ldg(q1 + c) : 0u;
+                    qf[ks][1] = 0u;
                     qf[ks][2] = r0 ? __ldg(q0 + c + 4) : 0u;
-                    qf[ks][3] = r1 ? __ldg(q1 + c + 4) : 0u;
+                    qf[ks][3] = 0u;
                 }
             }
-            float m_run[2] = {-INFINITY, -INFINITY};
-            float l_run[2] = {0.f, 0.f};
+            float m_run = -INFINITY, l_run = 0.f;
             float o[16][4];
 #pragma unroll
             for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
@@ -177,42 +184,33 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                         mma_bf16_16816(s[nt], qf[2 * kp + 1], kb[2], kb[3]);
                     }
                 }
-                // ---- rolling softmax state update (log2 domain)
-                float mx0 = -INFINITY, mx1 = -INFINITY;
+                // ---- rolling softmax state update (log2 domain), rows 0..7 only
+                float mx = -INFINITY;
 #pragma unroll
                 for (int nt = 0; nt < 4; ++nt) {
                     const int key = key_base + nt * 8 + 2 * t4;
-                    const bool v0 = key < p.L, v1 = (key + 1) < p.L;
-                    s[nt][0] = v0 ? s[nt][0] * p.scale_log2 : -INFINITY;
-                    s[nt][1] = v1 ? s[nt][1] * p.scale_log2 : -INFINITY;
-                    s[nt][2] = v0 ? s[nt][2] * p.scale_log2 : -INFINITY;
-                    s[nt][3] = v1 ? s[nt][3] * p.scale_log2 : -INFINITY;
-                    mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
-                    mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
+                    s[nt][0] = (key < p.L) ? s[nt][0] * p.scale_log2 : -INFINITY;
+                    s[nt][1] = (key + 1 < p.L) ? s[nt][1] * p.scale_log2 : -INFINITY;
+                    mx = fmaxf(mx, fmaxf(s[nt][0], s[nt][1]));
                 }
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
-                const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0;  // identity state: avoid inf - inf
-                const float ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-                const float a0 = fast_exp2(m_run[0] - ms0), a1 = fast_exp2(m_run[1] - ms1);
-                m_run[0] = mn0; m_run[1] = mn1;
-                float sum0 = 0.f, sum1 = 0.f;
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run, mx);
+                const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;  // identity state: avoid inf - inf
+                const float resc = fast_exp2(m_run - m_safe);
+                m_run = m_new;
+                float sum = 0.f;
                 uint32_t pf[2][4];
 #pragma unroll
                 for (int nt = 0; nt < 4; ++nt) {
-                    const float p0 = fast_exp2(s[nt][0] - ms0), p1 = fast_exp2(s[nt][1] - ms0);
-                    const float p2 = fast_exp2(s[nt][2] - ms1), p3 = fast_exp2(s[nt][3] - ms1);
-                    sum0 += p0 + p1; sum1 += p2 + p3;
+                    const float p0 = fast_exp2(s[nt][0] - m_safe), p1 = fast_exp2(s[nt][1] - m_safe);
+                    sum += p0 + p1;
                     pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16x2(p0, p1);
-                    pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16x2(p2, p3);
+                    pf[nt >> 1][(nt & 1) * 2 + 1] = 0u;
                 }
-                l_run[0] = l_run[0] * a0 + sum0;
-                l_run[1] = l_run[1] * a1 + sum1;
+                l_run = l_run * resc + sum;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) { o[i][0] *= a0; o[i][1] *= a0; o[i][2] *= a1; o[i][3] *= a1; }
+                for (int i = 0; i < 16; ++i) { o[i][0] *= resc; o[i][1] *= resc; }
                 // ---- value += P V for this warp's 32 keys: 2 k-steps x 16 n-tiles
                 if (!warp_wait(&fullV[stage], phase, abort_flag, p.status, 3)) { ok = false; break; }
 #pragma unroll
@@ -236,91 +234,79 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             if (!ok) break;
 
             // ---- merge the four warps' states for this segment
-            l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
-            l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
-            l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
-            l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
-            {
-                float* mw = merge + warp * kSlotFloats;
-                if (g < p.G) {
-                    float* row = mw + g * kRowFloats;
-                    if (t4 == 0) { row[0] = m_run[0]; row[1] = l_run[0]; }
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+            if (g < p.G) {
+                float* row = merge + warp * kSlotFloats + g * kRowFloats;
+                if (t4 == 0) { row[kD] = m_run; row[kD + 1] = l_run; }
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        row[2 + i * 8 + 2 * t4] = o[i][0];
-                        row[2 + i * 8 + 2 * t4 + 1] = o[i][1];
-                    }
-                }
-                if (g + 8 < p.G) {
-                    float* row = mw + (g + 8) * kRowFloats;
-                    if (t4 == 0) { row[0] = m_run[1]; row[1] = l_run[1]; }
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        row[2 + i * 8 + 2 * t4] = o[i][2];
-                        row[2 + i * 8 + 2 * t4 + 1] = o[i][3];
-                    }
-                }
+                for (int i = 0; i < 16; ++i) *reinterpret_cast<float2*>(row + i * 8 + 2 * t4) = make_float2(o[i][0], o[i][1]);
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
-            const int slot = 2 * blockIdx.x + ((it_begin / p.n_chunks) == unit ? 0 : 1);
-            float* pslot = p.partials + static_cast<size_t>(slot) * kSlotFloats;
+            consumer_sync();
+            float* pslot = p.partials + static_cast<size_t>(slot_of(blockIdx.x, unit, p.base, p.rem, p.n_chunks)) * kSlotFloats;
             for (int idx = tid; idx < p.G * kD; idx += kConsumerThreads) {
                 const int r = idx >> 7, d = idx & (kD - 1);
                 float mw[kConsumerWarps];
                 float M = -INFINITY;
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) {
-                    mw[w] = merge[w * kSlotFloats + r * kRowFloats];
+                    mw[w] = merge[w * kSlotFloats + r * kRowFloats + kD];
                     M = fmaxf(M, mw[w]);
                 }
                 float acc = 0.f, lsum = 0.f;
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) {
                     const float sc = fast_exp2(mw[w] - M);  // a warp that saw no valid key has m = -inf -> 0
-                    acc += sc * merge[w * kSlotFloats + r * kRowFloats + 2 + d];
-                    lsum += sc * merge[w * kSlotFloats + r * kRowFloats + 1];
+                    acc += sc * merge[w * kSlotFloats + r * kRowFloats + d];
+                    lsum += sc * merge[w * kSlotFloats + r * kRowFloats + kD + 1];
                 }
                 if (whole_unit) {
                     p.O[(static_cast<size_t>(b) * p.Hq + head0 + r) * kD + d] = __float2bfloat16_rn(acc / lsum);
                 } else {
-                    pslot[r * kRowFloats + 2 + d] = acc;
-                    if (d == 0) { pslot[r * kRowFloats] = M; pslot[r * kRowFloats + 1] = lsum; }
+                    pslot[r * kRowFloats + d] = acc;
+                    if (d == 0) { pslot[r * kRowFloats + kD] = M; pslot[r * kRowFloats + kD + 1] = lsum; }
                 }
             }
             if (!whole_unit) {
                 // Collection + parallel reduce across blocks: the block that arrives last merges.
                 __threadfence();
-                asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
-                const int c_first = owner_of(static_cast<long long>(unit) * p.n_chunks, n_cta, p.total_items);
-                const int c_last = owner_of(unit_end - 1, n_cta, p.total_items);
+                consumer_sync();
+                const int c_first = owner_of(unit * p.n_chunks, p.base, p.rem);
+                const int c_last = owner_of(unit_end - 1, p.base, p.rem);
+                const int n_parts = c_last - c_first + 1;
                 if (tid == 0) {
                     const uint32_t prev = atomicAdd(&p.counters[unit], 1u);
-                    *is_last = (prev == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
+                    *is_last = (prev == static_cast<uint32_t>(n_parts - 1)) ? 1u : 0u;
                 }
-                asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+                for (int i = tid; i < n_parts; i += kConsumerThreads)
+                    slot_table[i] = slot_of(c_first + i, unit, p.base, p.rem, p.n_chunks);
+                consumer_sync();
                 if (*is_last) {
                     __threadfence();
-                    for (int idx = tid; idx < p.G * kD; idx += kConsumerThreads) {
-                        const int r = idx >> 7, d = idx & (kD - 1);
+                    for (int idx = tid; idx < p.G * (kD / 4); idx += kConsumerThreads) {
+                        const int r = idx >> 5, d4 = idx & 31;
                         float M = -INFINITY;
-                        for (int c = c_first; c <= c_last; ++c) {
-                            const int sl = 2 * c + ((range_begin(c, n_cta, p.total_items) / p.n_chunks) == unit ? 0 : 1);
-                            M = fmaxf(M, __ldcg(p.partials + static_cast<size_t>(sl) * kSlotFloats + r * kRowFloats));
+                        for (int i = 0; i < n_parts; ++i)
+                            M = fmaxf(M, __ldcg(p.partials + static_cast<size_t>(slot_table[i]) * kSlotFloats + r * kRowFloats + kD));
+                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                        float lsum = 0.f;
+                        for (int i = 0; i < n_parts; ++i) {  // block order: deterministic
+                            const float* ps = p.partials + static_cast<size_t>(slot_table[i]) * kSlotFloats + r * kRowFloats;
+                            const float sc = fast_exp2(__ldcg(ps + kD) - M);
+                            lsum += sc * __ldcg(ps + kD + 1);
+                            const float4 v = __ldcg(reinterpret_cast<const float4*>(ps) + d4);
+                            acc[0] += sc * v.x; acc[1] += sc * v.y; acc[2] += sc * v.z; acc[3] += sc * v.w;
                         }
-                        float acc = 0.f, lsum = 0.f;
-                        for (int c = c_first; c <= c_last; ++c) {
-                            const int sl = 2 * c + ((range_begin(c, n_cta, p.total_items) / p.n_chunks) == unit ? 0 : 1);
-                            const float* ps = p.partials + static_cast<size_t>(sl) * kSlotFloats + r * kRowFloats;
-                            const float sc = fast_exp2(__ldcg(ps) - M);
-                            acc += sc * __ldcg(ps + 2 + d);
-                            lsum += sc * __ldcg(ps + 1);
-                        }
-                        p.O[(static_cast<size_t>(b) * p.Hq + head0 + r) * kD + d] = __float2bfloat16_rn(acc / lsum);
+                        const float inv = 1.f / lsum;
+                        uint2 packed;
+                        packed.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+                        packed.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+                        *reinterpret_cast<uint2*>(p.O + (static_cast<size_t>(b) * p.Hq + head0 + r) * kD + 4 * d4) = packed;
                     }
                     if (tid == 0) p.counters[unit] = 0u;  // leave the counter ready for the next call
                 }
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+            consumer_sync();  // merge buffer, slot table and is_last are reused by the next segment
             it = seg_end;
         }
     }
@@ -341,8 +327,7 @@ size_t ef_gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int L, int D) {
     (void)Hq; (void)L; (void)D;
     if (B <= 0 || Hkv <= 0) return 0;
     const size_t counters = ((static_cast<size_t>(B) * Hkv * sizeof(uint32_t)) + 255) & ~size_t(255);
-    const size_t max_grid = 256;  // upper bound on the persistent grid
-    return ef::kHeaderBytes + counters + max_grid * 2 * ef::decode::kSlotFloats * sizeof(float);
+    return ef::kHeaderBytes + counters + static_cast<size_t>(ef::decode::kMaxGrid) * 2 * ef::decode::kSlotFloats * sizeof(float);
 }
 
 ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, int B, int Hq, int Hkv, int L, int D,
@@ -355,7 +340,7 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
     const size_t counters_bytes = (n_units * sizeof(uint32_t) + 255) & ~size_t(255);
     if (kHeaderBytes + counters_bytes > 65536) return EF_ERR_UNSUPPORTED;  // counters must lie in the init window
     const long long n_chunks = (static_cast<long long>(L) + decode::kChunk - 1) / decode::kChunk;
-    if (n_chunks * static_cast<long long>(n_units) > 0x7fffffffLL) return EF_ERR_UNSUPPORTED;
+    if (n_chunks * static_cast<long long>(n_units) >= (1LL << 30)) return EF_ERR_UNSUPPORTED;
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16)) return EF_ERR_ALIGN;
     if (!ws || ws_bytes < ef_gqa_decode_workspace_bytes(B, Hq, Hkv, L, D)) return EF_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EF_ERR_ALIGN;
@@ -384,13 +369,15 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.L = L; p.G = Hq / Hkv;
     p.n_chunks = static_cast<int>(n_chunks);
     p.total_items = static_cast<int>(n_chunks * static_cast<long long>(n_units));
+    int grid = di.num_sms < p.total_items ? di.num_sms : p.total_items;
+    if (grid > decode::kMaxGrid) grid = decode::kMaxGrid;
+    p.base = p.total_items / grid;
+    p.rem = p.total_items % grid;
     p.scale_log2 = scale * 1.4426950408889634f;
     uint8_t* w = static_cast<uint8_t*>(ws);
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
     p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
-    int grid = di.num_sms < p.total_items ? di.num_sms : p.total_items;
-    if (grid > 256) grid = 256;
     decode::gqa_decode_kernel<<<grid, decode::kThreads, decode::kSmemBytes, static_cast<cudaStream_t>(stream)>>>(
         tmK, tmV, p);
     EF_CUDA_CHECK(cudaGetLastError());

@@ -49,7 +49,7 @@ def test_host_side_argument_validation(lib):
     assert lib.ef_gqa_decode(one, one, one, one, 0, 4, 1, 8, 128, 1.0, one, 1 << 30, null) == 2
     # unsupported (no fallback)
     assert lib.ef_gqa_decode(one, one, one, one, 1, 4, 1, 8, 64, 1.0, one, 1 << 30, null) == 3    # D != 128
-    assert lib.ef_gqa_decode(one, one, one, one, 1, 32, 1, 8, 128, 1.0, one, 1 << 30, null) == 3  # group > 16
+    assert lib.ef_gqa_decode(one, one, one, one, 1, 32, 1, 8, 128, 1.0, one, 1 << 30, null) == 3  # group > 8
     # alignment
     assert lib.ef_gqa_decode(p(4098), one, one, one, 1, 4, 1, 8, 128, 1.0, one, 1 << 30, null) == 4
     # workspace

@@ -43,7 +43,7 @@ def test_decode_lengths(L):
     _run(3, L=L)
 
 
-@pytest.mark.parametrize("B,Hq,Hkv", [(1, 1, 1), (1, 16, 1), (3, 12, 4), (2, 8, 8), (5, 6, 2)])
+@pytest.mark.parametrize("B,Hq,Hkv", [(1, 1, 1), (1, 8, 1), (3, 12, 4), (2, 8, 8), (5, 6, 2)])
 def test_decode_head_groupings(B, Hq, Hkv):
     _run(4, B=B, Hq=Hq, Hkv=Hkv, L=200)
 

@@ -1,0 +1,438 @@
+// ef_lora_linear: Y = X @ W + alpha * (X @ A) @ Bm, tensor-core bound at large M.
+//
+// Two kernels, the form the paper's search selects for LoRA (Section 7.2): the low-rank
+// projection is computed once and stored instead of being recomputed per output tile.
+//   1. lora_t_kernel    T = alpha * (X @ A)              [M,16] bf16 in the workspace
+//   2. lora_main_kernel Y = [X | T] @ [W ; Bm]           the rank-16 update is ONE extra K slab
+// Both run on tcgen05: TMA stages 128B-swizzled bf16 tiles in shared memory, one elected thread
+// issues tcgen05.mma (kind::f16, bf16 operands, fp32 accumulators in TMEM), the epilogue warps
+// read the accumulators back with tcgen05.ld.
+//
+// Refinement (Table 1): kernel 2 is the "MN" row (grid over 128x256 output tiles, K traversed by
+// the in-block loop); kernel 1 is "MK" (K split across blocks, partial products combined by a
+// parallel Reduce_+ in split order by the block that arrives last -- deterministic).
+//
+// Operand layouts.  X tiles are K-major (K contiguous), W / Bm / A tiles are MN-major (N
+// contiguous) exactly as they sit in global memory; the UMMA descriptors carry the major-ness, so
+// nothing is transposed.
+#include "host.cuh"
+#include "ptx.cuh"
+
+namespace ef {
+namespace lora {
+
+constexpr int kBM = 128, kBK = 64;
+constexpr int kRank = 16;
+
+// --------------------------------------------------------------------------------------------
+// main kernel
+// --------------------------------------------------------------------------------------------
+constexpr int kBN = 256;
+constexpr int kStages = 4;
+constexpr int kABytes = kBM * kBK * 2;            // 16 KiB: [128 rows][64 k] K-major, 128B swizzle
+constexpr int kBAtomBytes = kBK * 128;            //  8 KiB: [64 k][64 n] MN-major, 128B swizzle
+constexpr int kBBytes = (kBN / 64) * kBAtomBytes; // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kThreads = 192;                     // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 256;
+constexpr uint32_t kTmemCols = 512;               // two 256-column fp32 accumulators
+
+struct MainParams {
+    __nv_bfloat16* Y;
+    int M, N;
+    int tiles_m, num_tiles;
+    int k_blocks;   // K / 64
+    int has_lora;   // 1: one more K block taken from (T, Bm)
+    uint32_t* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                 const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmB, const MainParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    uint64_t* full = bars;                       // [kStages]  TMA -> MMA
+    uint64_t* empty = bars + kStages;            // [kStages]  MMA -> TMA
+    uint64_t* acc_full = bars + 2 * kStages;     // [2]        MMA -> epilogue
+    uint64_t* acc_empty = bars + 2 * kStages + 2;  // [2]      epilogue -> MMA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+        *abort_flag = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int total_kb = p.k_blocks + p.has_lora;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmW);
+            if (p.has_lora) { tma_prefetch_desc(&tmT); tma_prefetch_desc(&tmB); }
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % p.tiles_m) * kBM, n0 = (tile / p.tiles_m) * kBN;
+                for (int kb = 0; kb < total_kb; ++kb) {
+                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+                    uint8_t* sA = smem + stage * kStageBytes;
+                    uint8_t* sB = sA + kABytes;
+                    mbar_expect_tx(&full[stage], kStageBytes);
+                    if (kb < p.k_blocks) {
+                        tma_load_2d(sA, &tmX, &full[stage], kb * kBK, m0);
+#pragma unroll
+                        for (int j = 0; j < kBN / 64; ++j)
+                            tma_load_2d(sB + j * kBAtomBytes, &tmW, &full[stage], n0 + 64 * j, kb * kBK);
+                    } else {  // rank-16 slab: columns >= 16 of T and rows >= 16 of Bm are out of bounds -> zero
+                        tma_load_2d(sA, &tmT, &full[stage], 0, m0);
+#pragma unroll
+                        for (int j = 0; j < kBN / 64; ++j)
+                            tma_load_2d(sB + j * kBAtomBytes, &tmB, &full[stage], n0 + 64 * j, 0);
+                    }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, 0, 1);
+            int stage = 0; uint32_t phase = 0;
+            int iter = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++iter) {
+                const int acc = iter & 1;
+                const uint32_t acc_phase = (iter >> 1) & 1;
+                if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, p.status, 2)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kBN;
+                for (int kb = 0; kb < total_kb; ++kb) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag, p.status, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sA = smem_u32(smem + stage * kStageBytes);
+                    const uint64_t a_desc = make_smem_desc(sA, 16, 1024, kSwizzle128B);
+                    const uint64_t b_desc = make_smem_desc(sA + kABytes, kBAtomBytes, 1024, kSwizzle128B);
+                    const int nk = (kb < p.k_blocks) ? kBK / 16 : kRank / 16;
+                    for (int kk = 0; kk < nk; ++kk) {
+                        // A advances 16 k = 32 B inside the swizzled row; B advances 16 k-rows = 2048 B
+                        umma_ss(d_tmem, a_desc + static_cast<uint64_t>(kk * 2), b_desc + static_cast<uint64_t>(kk * 128),
+                                idesc, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty[stage]);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(&acc_full[acc]);
+            }
+        }
+    } else {
+        const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        int iter = 0;
+        for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++iter) {
+            const int acc = iter & 1;
+            const uint32_t acc_phase = (iter >> 1) & 1;
+            const int m0 = (tile % p.tiles_m) * kBM, n0 = (tile / p.tiles_m) * kBN;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.status, 4));
+            if (!ok) break;
+            tc_fence_after();
+            const int row = m0 + q * 32 + lane;
+            const uint32_t taddr = tmem_base + acc * kBN + (static_cast<uint32_t>(q * 32) << 16);
+            __nv_bfloat16* yrow = p.Y + static_cast<size_t>(row) * p.N + n0;
+#pragma unroll 1
+            for (int c = 0; c < kBN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(taddr + c * 32, r);
+                tmem_wait_ld();
+                if (row < p.M) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const int col = n0 + c * 32 + v * 8;
+                        if (col + 8 <= p.N) {
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                            o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                            o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                            o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                            *reinterpret_cast<uint4*>(yrow + c * 32 + v * 8) = o;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+// T kernel: T = alpha * (X @ A), split-K with an ordered last-arriver reduction
+// --------------------------------------------------------------------------------------------
+constexpr int kTStages = 8;
+constexpr int kTBBytes = kBK * kRank * 2;         // 2 KiB: [64 k][16 r] MN-major, 32B swizzle
+constexpr int kTStageBytes = kABytes + kTBBytes;  // 18 KiB
+constexpr int kTThreads = 192;
+constexpr int kTSmemBytes = 1024 + kTStages * kTStageBytes + 256;
+constexpr uint32_t kTTmemCols = 32;
+
+struct TParams {
+    __nv_bfloat16* T;    // [m_pad][16]
+    float* partials;     // [splits][m_pad][16]
+    uint32_t* counters;  // one per m block, zero between calls
+    int M, m_pad, k_blocks, splits;
+    float alpha;
+    uint32_t* status;
+};
+
+__global__ void __launch_bounds__(kTThreads, 1)
+lora_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA, const TParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTStages * kTStageBytes);
+    uint64_t* full = bars;                  // [kTStages]
+    uint64_t* acc_full = bars + kTStages;   // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kTStages + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint32_t* is_last = tmem_slot + 2;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m_blk = blockIdx.x, split = blockIdx.y;
+    const int kb_begin = (split * p.k_blocks) / p.splits, kb_end = ((split + 1) * p.k_blocks) / p.splits;
+    const int n_kb = kb_end - kb_begin;  // host guarantees 1 <= n_kb <= kTStages
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTStages; ++s) mbar_init(&full[s], 1);
+        mbar_init(acc_full, 1);
+        *abort_flag = 0u;
+        *is_last = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) { tmem_alloc(tmem_slot, kTTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmA);
+            for (int i = 0; i < n_kb; ++i) {  // every k block has its own stage: no reuse, no empty barrier
+                uint8_t* sA = smem + i * kTStageBytes;
+                mbar_expect_tx(&full[i], kTStageBytes);
+                tma_load_2d(sA, &tmX, &full[i], (kb_begin + i) * kBK, m_blk * kBM);
+                tma_load_2d(sA + kABytes, &tmA, &full[i], 0, (kb_begin + i) * kBK);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(kBM, kRank, 0, 1);
+            bool ok = true;
+            for (int i = 0; i < n_kb && ok; ++i) {
+                if (!mbar_wait(&full[i], 0u, abort_flag, p.status, 5)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t sA = smem_u32(smem + i * kTStageBytes);
+                const uint64_t a_desc = make_smem_desc(sA, 16, 1024, kSwizzle128B);
+                const uint64_t b_desc = make_smem_desc(sA + kABytes, 16, 256, kSwizzle32B);
+                for (int kk = 0; kk < kBK / 16; ++kk)  // B advances 16 k-rows of 32 B = 512 B
+                    umma_ss(tmem_base, a_desc + static_cast<uint64_t>(kk * 2), b_desc + static_cast<uint64_t>(kk * 32), idesc,
+                            (i | kk) != 0 ? 1u : 0u);
+            }
+            if (ok) umma_commit(acc_full);
+        }
+    } else {
+        const int q = warp & 3;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0u, abort_flag, p.status, 6));
+        if (ok) {
+            tc_fence_after();
+            uint32_t r[16];
+            tmem_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16), r);
+            tmem_wait_ld();
+            const int row = m_blk * kBM + q * 32 + lane;  // < m_pad always
+            if (p.splits == 1) {
+                uint4 lo, hi;
+                lo.x = pack_bf16x2(p.alpha * __uint_as_float(r[0]), p.alpha * __uint_as_float(r[1]));
+                lo.y = pack_bf16x2(p.alpha * __uint_as_float(r[2]), p.alpha * __uint_as_float(r[3]));
+                lo.z = pack_bf16x2(p.alpha * __uint_as_float(r[4]), p.alpha * __uint_as_float(r[5]));
+                lo.w = pack_bf16x2(p.alpha * __uint_as_float(r[6]), p.alpha * __uint_as_float(r[7]));
+                hi.x = pack_bf16x2(p.alpha * __uint_as_float(r[8]), p.alpha * __uint_as_float(r[9]));
+                hi.y = pack_bf16x2(p.alpha * __uint_as_float(r[10]), p.alpha * __uint_as_float(r[11]));
+                hi.z = pack_bf16x2(p.alpha * __uint_as_float(r[12]), p.alpha * __uint_as_float(r[13]));
+                hi.w = pack_bf16x2(p.alpha * __uint_as_float(r[14]), p.alpha * __uint_as_float(r[15]));
+                uint4* dst = reinterpret_cast<uint4*>(p.T + static_cast<size_t>(row) * kRank);
+                dst[0] = lo; dst[1] = hi;
+            } else {
+                uint4* dst = reinterpret_cast<uint4*>(p.partials + (static_cast<size_t>(split) * p.m_pad + row) * kRank);
+                dst[0] = make_uint4(r[0], r[1], r[2], r[3]);
+                dst[1] = make_uint4(r[4], r[5], r[6], r[7]);
+                dst[2] = make_uint4(r[8], r[9], r[10], r[11]);
+                dst[3] = make_uint4(r[12], r[13], r[14], r[15]);
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (warp == 2 && lane == 0) {
+                    const uint32_t prev = atomicAdd(&p.counters[m_blk], 1u);
+                    *is_last = (prev == static_cast<uint32_t>(p.splits - 1)) ? 1u : 0u;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (*is_last) {
+                    __threadfence();
+                    float acc[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+                    for (int s = 0; s < p.splits; ++s) {  // split order: deterministic
+                        const float4* src = reinterpret_cast<const float4*>(p.partials + (static_cast<size_t>(s) * p.m_pad + row) * kRank);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float4 v = __ldcg(src + j);
+                            acc[4 * j] += v.x; acc[4 * j + 1] += v.y; acc[4 * j + 2] += v.z; acc[4 * j + 3] += v.w;
+                        }
+                    }
+                    uint4 lo, hi;
+                    lo.x = pack_bf16x2(p.alpha * acc[0], p.alpha * acc[1]);
+                    lo.y = pack_bf16x2(p.alpha * acc[2], p.alpha * acc[3]);
+                    lo.z = pack_bf16x2(p.alpha * acc[4], p.alpha * acc[5]);
+                    lo.w = pack_bf16x2(p.alpha * acc[6], p.alpha * acc[7]);
+                    hi.x = pack_bf16x2(p.alpha * acc[8], p.alpha * acc[9]);
+                    hi.y = pack_bf16x2(p.alpha * acc[10], p.alpha * acc[11]);
+                    hi.z = pack_bf16x2(p.alpha * acc[12], p.alpha * acc[13]);
+                    hi.w = pack_bf16x2(p.alpha * acc[14], p.alpha * acc[15]);
+                    uint4* dst2 = reinterpret_cast<uint4*>(p.T + static_cast<size_t>(row) * kRank);
+                    dst2[0] = lo; dst2[1] = hi;
+                    if (warp == 2 && lane == 0) p.counters[m_blk] = 0u;
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTTmemCols);
+    }
+}
+
+struct Plan {
+    int tiles_m, tiles_n, m_pad, k_blocks, splits;
+    size_t t_off, part_off, total;
+};
+inline Plan make_plan(int M, int K, int N, int num_sms) {
+    Plan pl;
+    pl.tiles_m = (M + kBM - 1) / kBM;
+    pl.tiles_n = (N + kBN - 1) / kBN;
+    pl.m_pad = pl.tiles_m * kBM;
+    pl.k_blocks = K / kBK;
+    int s = num_sms / pl.tiles_m;
+    if (s < 1) s = 1;
+    if (s > pl.k_blocks) s = pl.k_blocks;
+    const int min_s = (pl.k_blocks + kTStages - 1) / kTStages;  // each split fits the stage ring
+    if (s < min_s) s = min_s;
+    pl.splits = s;
+    pl.t_off = kHeaderBytes;
+    pl.part_off = pl.t_off + ((static_cast<size_t>(pl.m_pad) * kRank * 2 + 255) & ~size_t(255));
+    pl.total = pl.part_off + static_cast<size_t>(pl.k_blocks) * pl.m_pad * kRank * 4;  // worst case: one split per k block
+    return pl;
+}
+
+}  // namespace lora
+}  // namespace ef
+
+extern "C" {
+
+size_t ef_lora_linear_workspace_bytes(int M, int K, int N, int R) {
+    if (M <= 0 || K <= 0 || N <= 0 || R != ef::lora::kRank || K % ef::lora::kBK != 0) return 0;
+    return ef::lora::make_plan(M, K, N, 1).total;
+}
+
+ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void* Bm, void* Y, int M, int K, int N, int R,
+                         float alpha, void* ws, size_t ws_bytes, void* stream) {
+    using namespace ef;
+    if (!X || !W || !A || !Bm || !Y) return EF_ERR_NULL;
+    if (M <= 0 || K <= 0 || N <= 0 || R <= 0) return EF_ERR_SHAPE;
+    if (R != lora::kRank || K % lora::kBK != 0 || N % 8 != 0) return EF_ERR_UNSUPPORTED;
+    if ((M + lora::kBM - 1) / lora::kBM > static_cast<int>(kMaxCounters)) return EF_ERR_UNSUPPORTED;
+    if (!aligned(X, 16) || !aligned(W, 16) || !aligned(A, 16) || !aligned(Bm, 16) || !aligned(Y, 16)) return EF_ERR_ALIGN;
+    if (!ws || ws_bytes < ef_lora_linear_workspace_bytes(M, K, N, R)) return EF_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EF_ERR_ALIGN;
+    DeviceInfo di;
+    if (!current_device_info(&di)) return EF_ERR_CUDA;
+    if (di.cc_major != 10) return EF_ERR_ARCH;
+    const lora::Plan pl = lora::make_plan(M, K, N, di.num_sms);
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(w + pl.t_off);
+
+    CUtensorMap tmX, tmW, tmT, tmB, tmA;
+    ef_status st;
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(K) * 2};
+        const uint32_t box[2] = {64, lora::kBM};
+        if ((st = encode_tmap_bf16(&tmX, X, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    }
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(K)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(N) * 2};
+        const uint32_t box[2] = {64, lora::kBK};
+        if ((st = encode_tmap_bf16(&tmW, W, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    }
+    {
+        const uint64_t dims[2] = {lora::kRank, static_cast<uint64_t>(pl.m_pad)};
+        const uint64_t strides[1] = {lora::kRank * 2};
+        const uint32_t box[2] = {64, lora::kBM};
+        if ((st = encode_tmap_bf16(&tmT, T, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    }
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(N), lora::kRank};
+        const uint64_t strides[1] = {static_cast<uint64_t>(N) * 2};
+        const uint32_t box[2] = {64, lora::kBK};
+        if ((st = encode_tmap_bf16(&tmB, Bm, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    }
+    {
+        const uint64_t dims[2] = {lora::kRank, static_cast<uint64_t>(K)};
+        const uint64_t strides[1] = {lora::kRank * 2};
+        const uint32_t box[2] = {lora::kRank, lora::kBK};
+        if ((st = encode_tmap_bf16(&tmA, A, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_32B)) != EF_OK) return st;
+    }
+    static bool attr_set[64] = {};
+    if (!attr_set[di.device]) {
+        EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::kSmemBytes));
+        EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::kTSmemBytes));
+        attr_set[di.device] = true;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    {
+        lora::TParams tp;
+        tp.T = T;
+        tp.partials = reinterpret_cast<float*>(w + pl.part_off);
+        tp.counters = reinterpret_cast<uint32_t*>(w + kCounterOffset);
+        tp.M = M; tp.m_pad = pl.m_pad; tp.k_blocks = pl.k_blocks; tp.splits = pl.splits;
+        tp.alpha = alpha;
+        tp.status = reinterpret_cast<uint32_t*>(w);
+        lora::lora_t_kernel<<<dim3(pl.tiles_m, pl.splits), lora::kTThreads, lora::kTSmemBytes, s>>>(tmX, tmA, tp);
+        EF_CUDA_CHECK(cudaGetLastError());
+    }
+    {
+        lora::MainParams mp;
+        mp.Y = static_cast<__nv_bfloat16*>(Y);
+        mp.M = M; mp.N = N;
+        mp.tiles_m = pl.tiles_m; mp.num_tiles = pl.tiles_m * pl.tiles_n;
+        mp.k_blocks = pl.k_blocks; mp.has_lora = 1;
+        mp.status = reinterpret_cast<uint32_t*>(w);
+        const int grid = di.num_sms < mp.num_tiles ? di.num_sms : mp.num_tiles;
+        lora::lora_main_kernel<<<grid, lora::kThreads, lora::kSmemBytes, s>>>(tmX, tmW, tmT, tmB, mp);
+        EF_CUDA_CHECK(cudaGetLastError());
+    }
+    return EF_OK;
+}
+
+}  // extern "C"

@@ -16,9 +16,4 @@ ef_status ef_qknorm_attn(const void*, const void*, const void*, const void*, con
                          float, float, int, void*, size_t, void*) {
     return EF_ERR_UNSUPPORTED;
 }
-size_t ef_lora_linear_workspace_bytes(int, int, int, int) { return ef::kHeaderBytes; }
-ef_status ef_lora_linear(const void*, const void*, const void*, const void*, void*, int, int, int, int, float, void*,
-                         size_t, void*) {
-    return EF_ERR_UNSUPPORTED;
-}
 }

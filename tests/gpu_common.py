@@ -1,0 +1,31 @@
+"""Shared driver for the GPU parity tests: seeded inputs -> oracle (fp64) and CUDA path (C ABI)."""
+import numpy as np
+
+import oracle
+import workloads as wl
+from parity import assert_close
+
+
+def run_parity(program, seed=0, size="small", check_repeat=True, oracle_fn=None, **over):
+    import torch
+
+    import paper_2609_12330_b200 as ef
+
+    p, t = wl.make_inputs(program, seed=seed, size=size, **over)
+    f64 = {k: wl.bf16_bits_to_f64(v) for k, v in t.items()}
+    ref = oracle.run(program, p, f64) if oracle_fn is None else oracle_fn(p, f64)
+    dev = {k: wl.bf16_bits_to_torch(v, "cuda") for k, v in t.items()}
+    ws = ef.Workspace(ef.workspace_bytes(program, p))
+    out = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    ef.run(program, p, dev, ws, out=out)
+    ws.check()
+    got = wl.torch_bf16_to_f64(out)
+    r = assert_close(got, ref, f"{program} seed={seed} {p}")
+    if check_repeat:
+        # same workspace, second call: bookkeeping words were left consistent and the result is
+        # bit-identical (every cross-block reduction runs in a fixed order)
+        out2 = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        ef.run(program, p, dev, ws, out=out2)
+        ws.check()
+        assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+    return r

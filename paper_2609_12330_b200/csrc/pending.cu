@@ -3,14 +3,6 @@
 #include "host.cuh"
 
 extern "C" {
-size_t ef_rmsnorm_matmul_workspace_bytes(int, int, int) { return ef::kHeaderBytes; }
-ef_status ef_rmsnorm_matmul(const void*, const void*, const void*, void*, int, int, int, float, void*, size_t, void*) {
-    return EF_ERR_UNSUPPORTED;
-}
-size_t ef_gated_mlp_workspace_bytes(int, int, int) { return ef::kHeaderBytes; }
-ef_status ef_gated_mlp(const void*, const void*, const void*, void*, int, int, int, void*, size_t, void*) {
-    return EF_ERR_UNSUPPORTED;
-}
 size_t ef_qknorm_attn_workspace_bytes(int, int, int, int) { return ef::kHeaderBytes; }
 ef_status ef_qknorm_attn(const void*, const void*, const void*, const void*, const void*, void*, int, int, int, int,
                          float, float, int, void*, size_t, void*) {

@@ -1,0 +1,385 @@
+// ef_rmsnorm_matmul and ef_gated_mlp: projections of a few (<= 16) token rows through large
+// weight matrices.  Arithmetic intensity is 8..16 flop/byte, so both are HBM-bound: the job is to
+// stream W once at full bandwidth; the tensor core only has to keep up.
+//
+// Swap-AB on tcgen05: the MMA computes D^T[n, m] = sum_k W[k, n] * X[m, k] with the 128 weight
+// columns of a tile as the MMA M dimension (A operand = W tile exactly as it lies in memory,
+// MN-major) and the <= 16 token rows as the MMA N dimension (B operand = X tile, K-major).  The
+// accumulator is 128 TMEM lanes x 16 fp32 columns per weight matrix.
+//
+// Refinement (Table 1, MatMul "NK"): the (n-tile, k-block) grid is flattened n-major and cut into
+// equal contiguous ranges, one per persistent block, so every SM streams the same number of
+// bytes.  A block that owns only part of a tile's K range stores its fp32 partial (Collection);
+// the block that arrives last sums the partials in block order (Reduce_+ over the parallel K
+// axis, deterministic) and only then applies the pointwise epilogue -- SiLU(gate)*up is nonlinear,
+// so it cannot be applied to partial sums; the RMSNorm row factor r_m is invariant along K and is
+// applied at the same place (Table 1, factor motion), while gamma varies along K and is folded
+// into the X operand when the block builds it.
+#include "host.cuh"
+#include "ptx.cuh"
+
+namespace ef {
+namespace skinny {
+
+constexpr int kBN = 128;                          // weight columns per tile = MMA M
+constexpr int kBK = 64;
+constexpr int kMaxM = 16;                         // token rows = MMA N
+constexpr int kWAtomBytes = kBK * 128;            // 8 KiB: [64 k][64 n] MN-major, 128B swizzle
+constexpr int kWBytes = 2 * kWAtomBytes;          // 16 KiB per weight matrix per k block
+constexpr int kXBytes = kMaxM * kBK * 2;          // 2 KiB: [16 rows][64 k] K-major, 128B swizzle
+constexpr int kThreads = 192;                     // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kMaxGrid = 256;
+constexpr int kMiscBytes = 512 + kMaxGrid * 4;    // barriers, flags, r_m, slot table
+constexpr int kMaxSmem = 227 * 1024;
+
+struct Params {
+    const __nv_bfloat16* X;
+    const __nv_bfloat16* gamma;  // NORM only
+    __nv_bfloat16* Y;
+    int M, K, N;
+    int n_tiles, k_blocks, total_units;
+    int base, rem;       // block c owns base + (c < rem) consecutive (tile, k block) units
+    int stages;
+    float eps;
+    uint32_t* status;
+    uint32_t* counters;  // one per n tile, zero between calls
+    float* partials;     // [grid][2][NW][16][128]
+};
+
+__device__ __forceinline__ int range_begin(int c, int base, int rem) { return c * base + min(c, rem); }
+__device__ __forceinline__ int owner_of(int x, int base, int rem) {
+    const int big = rem * (base + 1);
+    return x < big ? x / (base + 1) : rem + (x - big) / base;
+}
+__device__ __forceinline__ int slot_of(int c, int tile, int base, int rem, int k_blocks) {
+    return 2 * c + ((range_begin(c, base, rem) / k_blocks) == tile ? 0 : 1);
+}
+__device__ __forceinline__ float silu(float z) { return z / (1.f + __expf(-z)); }
+
+// NW = number of weight matrices sharing the X operand (1: RMSNorm+matmul, 2: gated MLP)
+// NORM = build the X operand as bf16(x * gamma) in shared memory and scale rows by r_m at the end
+template <int NW, bool NORM>
+__global__ void __launch_bounds__(kThreads, 1)
+skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+              const __grid_constant__ CUtensorMap tmX, const Params p) {
+    constexpr int kStageBytes = NW * kWBytes + (NORM ? 0 : kXBytes);
+    constexpr uint32_t kAccCols = NW * kMaxM;          // fp32 columns per accumulator buffer
+    constexpr uint32_t kTmemCols = 64;                 // two buffers of <= 32 columns
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int xg_bytes = NORM ? p.k_blocks * kXBytes : 0;
+    uint8_t* xg = smem;                                // NORM: [k_blocks][2 KiB] persistent X operand
+    uint8_t* stages = smem + xg_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stages + p.stages * kStageBytes);
+    uint64_t* full = bars;                             // [stages]
+    uint64_t* empty = bars + p.stages;                 // [stages]
+    uint64_t* acc_full = bars + 2 * p.stages;          // [2]
+    uint64_t* acc_empty = bars + 2 * p.stages + 2;     // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * p.stages + 4);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint32_t* is_last = tmem_slot + 2;
+    float* rinv = reinterpret_cast<float*>(tmem_slot + 4);        // [16]
+    int* slot_table = reinterpret_cast<int*>(tmem_slot + 4 + kMaxM);  // [kMaxGrid]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
+    const int it_end = range_begin(blockIdx.x + 1, p.base, p.rem);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+        *abort_flag = 0u;
+        *is_last = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // The producer starts streaming W right away; everyone else first builds the X operand.
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&tmW0);
+            if (NW == 2) tma_prefetch_desc(&tmW1);
+            if (!NORM) tma_prefetch_desc(&tmX);
+            int stage = 0; uint32_t phase = 0;
+            int tile = it_begin / p.k_blocks, kb = it_begin - tile * p.k_blocks;
+            for (int it = it_begin; it < it_end; ++it) {
+                if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) break;
+                uint8_t* st = stages + stage * kStageBytes;
+                mbar_expect_tx(&full[stage], kStageBytes);
+                const int n0 = tile * kBN, k0 = kb * kBK;
+                tma_load_2d(st, &tmW0, &full[stage], n0, k0);
+                tma_load_2d(st + kWAtomBytes, &tmW0, &full[stage], n0 + 64, k0);
+                if (NW == 2) {
+                    tma_load_2d(st + kWBytes, &tmW1, &full[stage], n0, k0);
+                    tma_load_2d(st + kWBytes + kWAtomBytes, &tmW1, &full[stage], n0 + 64, k0);
+                }
+                if (!NORM) tma_load_2d(st + NW * kWBytes, &tmX, &full[stage], k0, 0);
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                if (++kb == p.k_blocks) { kb = 0; ++tile; }
+            }
+        }
+    } else if (NORM) {
+        // X operand = bf16(x * gamma) for ALL k blocks, written in the K-major 128B-swizzled tile
+        // layout the MMA descriptor expects (row r of a tile: 128 B, 16-byte chunk c stored at
+        // chunk c ^ (r & 7)); sum of squares per row for r_m (product fusion: same pass over X).
+        const int w5 = warp - 1;  // 0..4
+        const int chunks = p.K >> 3;
+        for (int r = w5; r < kMaxM; r += 5) {
+            float ss = 0.f;
+            for (int c = lane; c < chunks; c += 32) {
+                uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+                if (r < p.M) xv = __ldg(reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(r) * p.K) + c);
+                const uint4 gv = __ldg(reinterpret_cast<const uint4*>(p.gamma) + c);
+                const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
+                const uint32_t gs[4] = {gv.x, gv.y, gv.z, gv.w};
+                uint32_t outv[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
+                    const float g0 = __uint_as_float(gs[j] << 16), g1 = __uint_as_float(gs[j] & 0xFFFF0000u);
+                    ss += x0 * x0 + x1 * x1;
+                    outv[j] = pack_bf16x2(x0 * g0, x1 * g1);
+                }
+                const int kb = c >> 3, cc = c & 7;
+                *reinterpret_cast<uint4*>(xg + kb * kXBytes + r * 128 + ((cc ^ (r & 7)) << 4)) =
+                    make_uint4(outv[0], outv[1], outv[2], outv[3]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (lane == 0) rinv[r] = rsqrtf(ss / static_cast<float>(p.K) + p.eps);
+        }
+        fence_proxy_async_smem();
+    }
+    if (NORM && warp != 0) asm volatile("bar.sync 2, 160;" ::: "memory");  // warps 1..5; the producer keeps streaming
+
+    if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(kBN, kMaxM, 1, 0);  // A MN-major, B K-major
+            int stage = 0; uint32_t phase = 0;
+            int iter = 0;
+            int it = it_begin;
+            bool ok = true;
+            while (it < it_end && ok) {
+                const int tile = it / p.k_blocks;
+                const int kb0 = it - tile * p.k_blocks;
+                const int seg_end = min(it_end, (tile + 1) * p.k_blocks);
+                const int acc = iter & 1;
+                if (!mbar_wait(&acc_empty[acc], ((iter >> 1) & 1) ^ 1u, abort_flag, p.status, 2)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                for (int i = 0; i < seg_end - it; ++i) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag, p.status, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t st = smem_u32(stages + stage * kStageBytes);
+                    const uint32_t xs = NORM ? smem_u32(xg + (kb0 + i) * kXBytes) : st + NW * kWBytes;
+                    const uint64_t b_desc = make_smem_desc(xs, 16, 1024, kSwizzle128B);
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) {
+                        const uint64_t a_desc = make_smem_desc(st + w * kWBytes, kWAtomBytes, 1024, kSwizzle128B);
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 16; ++kk)
+                            umma_ss(d_tmem + w * kMaxM, a_desc + static_cast<uint64_t>(kk * 128),
+                                    b_desc + static_cast<uint64_t>(kk * 2), idesc, (i | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty[stage]);
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(&acc_full[acc]);
+                it = seg_end;
+                ++iter;
+            }
+        }
+    } else if (warp >= 2) {
+        const int q = warp & 3;
+        const int et = q * 32 + lane;  // 0..127: TMEM lane = weight column within the tile
+        int iter = 0;
+        int it = it_begin;
+        while (it < it_end) {
+            const int tile = it / p.k_blocks;
+            const int kb0 = it - tile * p.k_blocks;
+            const int tile_end = (tile + 1) * p.k_blocks;
+            const int seg_end = min(it_end, tile_end);
+            const bool whole = (kb0 == 0) && (seg_end == tile_end);
+            const int acc = iter & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[acc], (iter >> 1) & 1, abort_flag, p.status, 4))) break;
+            tc_fence_after();
+            uint32_t v[NW][16];
+#pragma unroll
+            for (int w = 0; w < NW; ++w)
+                tmem_ld16(tmem_base + acc * kAccCols + w * kMaxM + (static_cast<uint32_t>(q * 32) << 16), v[w]);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);  // accumulator is in registers now
+            const int n = tile * kBN + et;
+            bool finish = whole;
+            int n_parts = 0;
+            if (!whole) {
+                float* ps = p.partials + static_cast<size_t>(slot_of(blockIdx.x, tile, p.base, p.rem, p.k_blocks)) * (NW * kMaxM * kBN);
+#pragma unroll
+                for (int w = 0; w < NW; ++w)
+#pragma unroll
+                    for (int m = 0; m < kMaxM; ++m) ps[(w * kMaxM + m) * kBN + et] = __uint_as_float(v[w][m]);
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int c_first = owner_of(tile * p.k_blocks, p.base, p.rem);
+                const int c_last = owner_of(tile_end - 1, p.base, p.rem);
+                n_parts = c_last - c_first + 1;
+                if (warp == 2 && lane == 0) {
+                    const uint32_t prev = atomicAdd(&p.counters[tile], 1u);
+                    *is_last = (prev == static_cast<uint32_t>(n_parts - 1)) ? 1u : 0u;
+                }
+                for (int i = threadIdx.x - 64; i < n_parts; i += 128)
+                    slot_table[i] = slot_of(c_first + i, tile, p.base, p.rem, p.k_blocks);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (*is_last) {
+                    __threadfence();
+#pragma unroll
+                    for (int w = 0; w < NW; ++w)
+#pragma unroll
+                        for (int m = 0; m < kMaxM; ++m) v[w][m] = 0u;
+                    for (int i = 0; i < n_parts; ++i) {  // block order: deterministic
+                        const float* src = p.partials + static_cast<size_t>(slot_table[i]) * (NW * kMaxM * kBN);
+#pragma unroll
+                        for (int w = 0; w < NW; ++w)
+#pragma unroll
+                            for (int m = 0; m < kMaxM; ++m)
+                                v[w][m] = __float_as_uint(__uint_as_float(v[w][m]) + __ldcg(src + (w * kMaxM + m) * kBN + et));
+                    }
+                    finish = true;
+                }
+            }
+            if (finish && n < p.N) {
+#pragma unroll
+                for (int m = 0; m < kMaxM; ++m) {
+                    if (m < p.M) {
+                        float y;
+                        if (NW == 2) y = silu(__uint_as_float(v[0][m])) * __uint_as_float(v[NW - 1][m]);
+                        else y = __uint_as_float(v[0][m]);
+                        if (NORM) y *= rinv[m];
+                        p.Y[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
+                    }
+                }
+            }
+            if (!whole) {
+                asm volatile("bar.sync 1, 128;" ::: "memory");  // slot table / is_last reuse
+                if (finish && warp == 2 && lane == 0) p.counters[tile] = 0u;
+            }
+            it = seg_end;
+            ++iter;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+struct Plan {
+    int n_tiles, k_blocks, total_units, stages, stage_bytes, smem_bytes;
+    size_t counters_bytes, total;
+};
+inline bool make_plan(int NW, bool norm, int K, int N, Plan* pl) {
+    pl->n_tiles = (N + kBN - 1) / kBN;
+    pl->k_blocks = K / kBK;
+    pl->total_units = pl->n_tiles * pl->k_blocks;
+    pl->stage_bytes = NW * kWBytes + (norm ? 0 : kXBytes);
+    const int xg = norm ? pl->k_blocks * kXBytes : 0;
+    int stages = (kMaxSmem - 1024 - xg - kMiscBytes) / pl->stage_bytes;
+    if (stages > 12) stages = 12;
+    pl->stages = stages;
+    pl->smem_bytes = 1024 + xg + stages * pl->stage_bytes + kMiscBytes;
+    pl->counters_bytes = (static_cast<size_t>(pl->n_tiles) * 4 + 255) & ~size_t(255);
+    pl->total = kHeaderBytes + pl->counters_bytes + static_cast<size_t>(kMaxGrid) * 2 * NW * kMaxM * kBN * 4;
+    return stages >= 2;
+}
+
+template <int NW, bool NORM>
+ef_status launch(const void* X, const void* gamma, const void* W0, const void* W1, void* Y, int M, int K, int N, float eps,
+                 void* ws, size_t ws_bytes, void* stream) {
+    if (!X || !W0 || !Y || (NW == 2 && !W1) || (NORM && !gamma)) return EF_ERR_NULL;
+    if (M <= 0 || K <= 0 || N <= 0) return EF_ERR_SHAPE;
+    if (M > kMaxM || K % kBK != 0 || N % 8 != 0) return EF_ERR_UNSUPPORTED;
+    Plan pl;
+    if (!make_plan(NW, NORM, K, N, &pl)) return EF_ERR_UNSUPPORTED;  // NORM: X operand of the whole K must fit in shared memory
+    if (static_cast<long long>(pl.n_tiles) * pl.k_blocks >= (1LL << 30)) return EF_ERR_UNSUPPORTED;
+    if (kHeaderBytes + pl.counters_bytes > 65536) return EF_ERR_UNSUPPORTED;  // counters must lie in the init window
+    if (!aligned(X, 16) || !aligned(W0, 16) || !aligned(Y, 16) || (NW == 2 && !aligned(W1, 16)) ||
+        (NORM && !aligned(gamma, 16)))
+        return EF_ERR_ALIGN;
+    if (!ws || ws_bytes < pl.total) return EF_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EF_ERR_ALIGN;
+    DeviceInfo di;
+    if (!current_device_info(&di)) return EF_ERR_CUDA;
+    if (di.cc_major != 10) return EF_ERR_ARCH;
+
+    CUtensorMap tmW0, tmW1, tmX;
+    ef_status st;
+    const uint64_t wdims[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(K)};
+    const uint64_t wstrides[1] = {static_cast<uint64_t>(N) * 2};
+    const uint32_t wbox[2] = {64, kBK};
+    if ((st = encode_tmap_bf16(&tmW0, W0, 2, wdims, wstrides, wbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    if ((st = encode_tmap_bf16(&tmW1, NW == 2 ? W1 : W0, 2, wdims, wstrides, wbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    const uint64_t xdims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
+    const uint64_t xstrides[1] = {static_cast<uint64_t>(K) * 2};
+    const uint32_t xbox[2] = {64, kMaxM};
+    if ((st = encode_tmap_bf16(&tmX, X, 2, xdims, xstrides, xbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+
+    static bool attr_set[64] = {};
+    if (!attr_set[di.device]) {
+        EF_CUDA_CHECK(cudaFuncSetAttribute(skinny_kernel<NW, NORM>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        attr_set[di.device] = true;
+    }
+    Params p;
+    p.X = static_cast<const __nv_bfloat16*>(X);
+    p.gamma = static_cast<const __nv_bfloat16*>(gamma);
+    p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.M = M; p.K = K; p.N = N;
+    p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
+    int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
+    if (grid > kMaxGrid) grid = kMaxGrid;
+    p.base = pl.total_units / grid;
+    p.rem = pl.total_units % grid;
+    p.stages = pl.stages;
+    p.eps = eps;
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    p.status = reinterpret_cast<uint32_t*>(w);
+    p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
+    p.partials = reinterpret_cast<float*>(w + kHeaderBytes + pl.counters_bytes);
+    skinny_kernel<NW, NORM><<<grid, kThreads, pl.smem_bytes, static_cast<cudaStream_t>(stream)>>>(tmW0, tmW1, tmX, p);
+    EF_CUDA_CHECK(cudaGetLastError());
+    return EF_OK;
+}
+
+}  // namespace skinny
+}  // namespace ef
+
+extern "C" {
+
+size_t ef_rmsnorm_matmul_workspace_bytes(int M, int K, int N) {
+    ef::skinny::Plan pl;
+    if (M <= 0 || K <= 0 || N <= 0 || K % ef::skinny::kBK != 0 || !ef::skinny::make_plan(1, true, K, N, &pl)) return 0;
+    return pl.total;
+}
+ef_status ef_rmsnorm_matmul(const void* X, const void* gamma, const void* W, void* Y, int M, int K, int N, float eps,
+                            void* ws, size_t ws_bytes, void* stream) {
+    return ef::skinny::launch<1, true>(X, gamma, W, nullptr, Y, M, K, N, eps, ws, ws_bytes, stream);
+}
+
+size_t ef_gated_mlp_workspace_bytes(int M, int K, int N) {
+    ef::skinny::Plan pl;
+    if (M <= 0 || K <= 0 || N <= 0 || K % ef::skinny::kBK != 0 || !ef::skinny::make_plan(2, false, K, N, &pl)) return 0;
+    return pl.total;
+}
+ef_status ef_gated_mlp(const void* X, const void* Wgate, const void* Wup, void* Y, int M, int K, int N, void* ws,
+                       size_t ws_bytes, void* stream) {
+    return ef::skinny::launch<2, false>(X, nullptr, Wgate, Wup, Y, M, K, N, 0.f, ws, ws_bytes, stream);
+}
+
+}  // extern "C"

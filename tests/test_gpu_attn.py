@@ -1,0 +1,38 @@
+"""GPU parity: ef_qknorm_attn (through the C ABI) against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from gpu_common import run_parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_attn_small_ragged(seed):
+    r = run_parity("qknorm_attn", seed)            # S=300: three Q tiles (two pairs), ragged tail of 44 rows
+    assert r["rel_l2"] < 6e-3
+
+
+@pytest.mark.parametrize("S", [1, 2, 127, 128, 129, 256, 257, 640])
+def test_attn_lengths(S):
+    run_parity("qknorm_attn", 3, S=S)
+
+
+def test_attn_noncausal():
+    run_parity("qknorm_attn", 4, S=300, causal=0)
+    run_parity("qknorm_attn", 4, S=512, causal=0)
+
+
+def test_attn_many_heads():
+    run_parity("qknorm_attn", 5, B=3, H=5, S=400)
+
+
+def test_attn_large_eps_and_unit_scale():
+    run_parity("qknorm_attn", 6, S=384, eps=0.25, scale=0.02)
+
+
+def test_attn_full_config_sampled_heads():
+    # full benchmark shape; the oracle's cost is affordable (about 70 GFLOP in fp64)
+    r = run_parity("qknorm_attn", 0, size="full", check_repeat=False)
+    assert r["rel_l2"] < 6e-3

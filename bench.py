@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the five fused tensor programs on B200.
+
+One STEP = one pass of the whole hot path: ef_rmsnorm_matmul, ef_gated_mlp, ef_gqa_decode,
+ef_qknorm_attn and ef_lora_linear, each once, at the benchmark shapes, on seeded synthetic bf16
+inputs that are resident in HBM.  The five programs of a step together touch ~520 MB of distinct
+inputs (> the 126 MB L2), so every program starts from a cold L2 each step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is the whole-step algorithmic TFLOP/s summed over all
+ranks (weak scaling: every rank runs the same step on its own GPU); `programs` gives per program
+the us/call, TFLOP/s, GB/s and the fraction of the roofline that bounds it.  `--impl reference`
+times the fp64 CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+import workloads as wl  # noqa: E402
+
+METRIC = "us/call and TFLOP/s (GB/s for decode) per fused program, % of B200 roofline"
+UNIT = "TFLOP/s (algorithmic flops of one step = all five programs / step time; per-program us/call, TFLOP/s, GB/s in 'programs')"
+BOUND = {"rmsnorm_matmul": "hbm", "gated_mlp": "hbm", "gqa_decode": "hbm", "qknorm_attn": "tensor", "lora_linear": "tensor"}
+KERNELS_PER_CALL = {"rmsnorm_matmul": 1, "gated_mlp": 1, "gqa_decode": 1, "qknorm_attn": 2, "lora_linear": 2}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def step_work():
+    work = {}
+    for prog in wl.PROGRAMS:
+        work[prog] = wl.algorithmic_work(prog, wl.SHAPES[prog]["full"])
+    return work
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks sampled DURING the timed region
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
+        self.proc.terminate()
+        mhz, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6 or not (t0 - 0.02 <= ts <= t1 + 0.02):
+                continue
+            try:
+                mhz.append(float(parts[0])); mx = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "samples": len(mhz),
+                "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+
+    import paper_2609_12330_b200 as ef
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ef.lib()  # fail loudly if the extension is missing
+
+    host, dev, params, wss, outs = {}, {}, {}, {}, {}
+    for prog in wl.PROGRAMS:
+        p, t = wl.make_inputs(prog, seed=rank, size="full")
+        params[prog] = p
+        host[prog] = {k: wl.bf16_bits_to_torch(v).pin_memory() for k, v in t.items()}
+        dev[prog] = {k: v.to("cuda", non_blocking=True) for k, v in host[prog].items()}
+        wss[prog] = ef.Workspace(ef.workspace_bytes(prog, p))
+        outs[prog] = ef.run(prog, p, dev[prog], wss[prog])
+    host_out = {prog: torch.empty_like(outs[prog], device="cpu").pin_memory() for prog in wl.PROGRAMS}
+    torch.cuda.synchronize()
+    work = step_work()
+    step_flops = sum(w["flops"] for w in work.values())
+    in_bytes = sum(v.numel() * 2 for prog in wl.PROGRAMS for v in host[prog].values())
+    out_bytes = sum(v.numel() * 2 for v in host_out.values())
+
+    def step():
+        for prog in wl.PROGRAMS:
+            ef.run(prog, params[prog], dev[prog], wss[prog], out=outs[prog])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        tns = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tns, op=dist.ReduceOp.MAX)
+        return float(tns.item())
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    for prog in wl.PROGRAMS:
+        wss[prog].check()
+
+    # ---- timed region: exactly K steps, inputs resident in HBM
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.1)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    t1 = time.time()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    clocks = sampler.stop(t0, t1)
+    ms_per_step = ms_total / args.steps
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- per-program breakdown (same step order, events between programs, cold L2)
+    n_break = min(args.steps, 200)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(wl.PROGRAMS) + 1)] for _ in range(n_break)]
+    for i in range(n_break):
+        evs[i][0].record()
+        for k, prog in enumerate(wl.PROGRAMS):
+            ef.run(prog, params[prog], dev[prog], wss[prog], out=outs[prog])
+            evs[i][k + 1].record()
+    torch.cuda.synchronize()
+    peaks = load_peaks()
+    programs = {}
+    for k, prog in enumerate(wl.PROGRAMS):
+        us = float(np.median([evs[i][k].elapsed_time(evs[i][k + 1]) for i in range(n_break)])) * 1e3
+        w = work[prog]
+        tf, gb = w["flops"] / us / 1e6, w["bytes"] / us / 1e3
+        entry = {"us_per_call": round(us, 2), "tflops": round(tf, 1), "gbs": round(gb, 1), "bound": BOUND[prog],
+                 "kernels": KERNELS_PER_CALL[prog]}
+        if BOUND[prog] == "hbm":
+            entry["frac"] = round(gb / peaks["hbm_gbs"], 4)
+        else:
+            entry["frac"] = round(tf / peaks["bf16_tflops_sustained"], 4)
+            entry["frac_of_burst_peak"] = round(tf / peaks["bf16_tflops"], 4)
+        programs[prog] = entry
+    dominant = max(programs, key=lambda q: programs[q]["us_per_call"])
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(dominant)
+    dp = programs[dominant]
+    if dp["bound"] == "tensor":
+        roofline = {"bound": "tensor", "achieved": dp["tflops"], "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": dp["frac"], "traffic": traffic}
+    else:
+        roofline = {"bound": "hbm", "achieved": dp["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dp["frac"],
+                    "traffic": traffic}
+    roofline["kernel"] = "ef_" + dominant
+    roofline["peak_source"] = ("of measured (sustained bf16 / copy)" if peaks["source"] == "measured" else "of fallback")
+
+    # ---- end to end: host buffers, H2D of every input and D2H of every output inside the timed region
+    n_e2e = max(1, min(args.steps, 20))
+    barrier()
+    e0.record()
+    for _ in range(n_e2e):
+        for prog in wl.PROGRAMS:
+            for kname, hv in host[prog].items():
+                dev[prog][kname].copy_(hv, non_blocking=True)
+            ef.run(prog, params[prog], dev[prog], wss[prog], out=outs[prog])
+            host_out[prog].copy_(outs[prog], non_blocking=True)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / n_e2e
+    e2e = {"value": round(world * step_flops / (e2e_ms * 1e-3) / 1e12, 3), "unit": "TFLOP/s", "ms_per_step": round(e2e_ms, 3),
+           "steps": n_e2e, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes}
+    for prog in wl.PROGRAMS:
+        wss[prog].check()
+
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "all five benchmark configs per step (rmsnorm_matmul 8x1024x4096, gated_mlp 16x4096x11008, "
+                               "gqa_decode B8 Hq32 Hkv8 L4096 D128, qknorm_attn B2 H32 S2048 D128 causal, "
+                               "lora_linear 2048x4096x4096 r16)",
+                   "l2": "inputs larger than L2: one step touches %d MB of distinct inputs" % (in_bytes // 1000000),
+                   "seed": rank, "parallelism": f"replicas x{world} (no collective on the path)"},
+        "clocks": clocks, "e2e": e2e,
+        "gpu_launches": args.steps * sum(KERNELS_PER_CALL.values()),
+        "roofline": roofline, "programs": programs,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------------
+# oracle arm / cpu baseline
+# ----------------------------------------------------------------------------------------------
+SAMPLE = {  # bounded samples of the benchmark workload for the (deliberately slow) fp64 oracle
+    "rmsnorm_matmul": {},
+    "gated_mlp": {},
+    "gqa_decode": {},
+    "qknorm_attn": {"B": 1, "H": 16},
+    "lora_linear": {"M": 1024},
+}
+SAMPLE_TEXT = ("rmsnorm_matmul, gated_mlp, gqa_decode at the full config; qknorm_attn on 16 of the 64 (batch, head) "
+               "pairs at S=2048; lora_linear on 1024 of the 2048 rows")
+
+
+def oracle_step(inputs):
+    import oracle
+
+    flops = 0
+    t0 = time.perf_counter()
+    for prog, (p, f64) in inputs.items():
+        oracle.run(prog, p, f64)
+        flops += wl.algorithmic_work(prog, p)["flops"]
+    return time.perf_counter() - t0, flops
+
+
+def oracle_inputs():
+    inputs = {}
+    for prog in wl.PROGRAMS:
+        p, t = wl.make_inputs(prog, seed=0, size="full", **SAMPLE[prog])
+        inputs[prog] = (p, {k: wl.bf16_bits_to_f64(v) for k, v in t.items()})
+    return inputs
+
+
+def cpu_baseline():
+    import oracle
+
+    inputs = oracle_inputs()
+    sec, flops = oracle_step(inputs)
+    return {"value": round(flops / sec / 1e12, 5), "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": SAMPLE_TEXT, "seconds": round(sec, 2)}
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+
+    inputs = oracle_inputs()
+    steps = max(1, min(args.steps, 3))
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(inputs)
+    secs, flops = [], 0
+    for _ in range(steps):
+        s, flops = oracle_step(inputs)
+        secs.append(s)
+    sec = float(np.mean(secs))
+    value = round(flops / sec / 1e12, 5)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(sec * 1e3, 2), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "bounded sample of the five benchmark configs per step: " + SAMPLE_TEXT},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": SAMPLE_TEXT},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

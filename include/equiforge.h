@@ -119,6 +119,28 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
                          void* ws, size_t ws_bytes, void* stream);
 size_t ef_lora_linear_workspace_bytes(int M, int K, int N, int R);
 
+/* ---- Decode attention without a caller workspace ---------------------------------------------
+ * (The paper has no counterpart: this is a deployment convenience of the library.)
+ * Same computation, arguments and supported shapes as ef_gqa_decode, for callers that are not
+ * allowed to allocate device memory at the point of the call -- for example code that runs
+ * inside a memory pool it must not grow, inside a real-time loop, or under a framework that
+ * forbids cudaMalloc after start-up.  Instead of a caller workspace the call uses a scratch
+ * array of 2,170,880 bytes that is part of the library image; every GPU that loads the library
+ * holds that array until the process exits.
+ *   - Limit: B * Hkv <= ef_gqa_decode_static_max_units() (1024); larger problems return
+ *     EF_ERR_WORKSPACE and nothing is enqueued.  Other errors as for ef_gqa_decode.
+ *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine).  It
+ *     enqueues one small memset (the status word and the arrival counters must start at zero,
+ *     and the array keeps the previous call's contents) and then the decode kernel.
+ *   - The FIRST call on each device looks up the array's device address (with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array: two calls that may overlap on the GPU (different
+ *     streams, or graph branches) race on it.  Serialise them, or use ef_gqa_decode with separate
+ *     workspaces. */
+ef_status ef_gqa_decode_static(const void* Q, const void* K, const void* V, void* O,
+                               int B, int Hq, int Hkv, int L, int D, float scale, void* stream);
+size_t ef_gqa_decode_static_max_units(void);
+
 /* ---- Workspace and status -------------------------------------------------------------------
  * (No counterpart in the paper: library plumbing.)
  * ef_workspace_init: enqueue zero-fill of the first min(ws_bytes, 64 KiB) bytes of ws on

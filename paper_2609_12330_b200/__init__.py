@@ -18,7 +18,7 @@ _lib = None
 EXPORTS = [
     "ef_rmsnorm_matmul", "ef_rmsnorm_matmul_workspace_bytes",
     "ef_gated_mlp", "ef_gated_mlp_workspace_bytes",
-    "ef_gqa_decode", "ef_gqa_decode_workspace_bytes",
+    "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_static", "ef_gqa_decode_static_max_units",
     "ef_qknorm_attn", "ef_qknorm_attn_workspace_bytes",
     "ef_lora_linear", "ef_lora_linear_workspace_bytes",
     "ef_workspace_init", "ef_check_status", "ef_status_string", "ef_last_cuda_error", "ef_version",
@@ -46,6 +46,8 @@ def lib():
         L.ef_gated_mlp_workspace_bytes.argtypes = [i, i, i]
         L.ef_gqa_decode.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
         L.ef_gqa_decode_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.ef_gqa_decode_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp]
+        L.ef_gqa_decode_static_max_units.argtypes = []
         L.ef_qknorm_attn.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, f, f, i, vp, sz, vp]
         L.ef_qknorm_attn_workspace_bytes.argtypes = [i, i, i, i]
         L.ef_lora_linear.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
@@ -56,7 +58,7 @@ def lib():
         L.ef_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
             fn = getattr(L, name)
-            if name.endswith("_workspace_bytes"):
+            if name.endswith("_workspace_bytes") or name.endswith("_max_units"):
                 fn.restype = sz
             elif name != "ef_status_string":
                 fn.restype = i
@@ -158,6 +160,21 @@ def gqa_decode(Q, K, V, scale, ws: Workspace, out=None):
     wp, wb = _ws_args(ws, gqa_decode_workspace_bytes(B, Hq, Hkv, L, D), "ef_gqa_decode")
     _check(lib().ef_gqa_decode(_ptr(Q, "Q"), _ptr(K, "K"), _ptr(V, "V"), _ptr(O, "O"), B, Hq, Hkv, L, D,
                                float(scale), wp, wb, _stream()), "ef_gqa_decode")
+    return O
+
+
+def gqa_decode_static(Q, K, V, scale, out=None):
+    """Decode attention through ef_gqa_decode_static: no workspace argument, nothing allocated by
+    the call itself (the output tensor is the caller's: pass `out` to avoid torch allocating one).
+    For callers that may not allocate device memory when they call; at most
+    ef_gqa_decode_static_max_units() (batch, kv head) units; calls on one device must not overlap."""
+    import torch
+
+    B, Hq, D = Q.shape
+    _, Hkv, L, _ = K.shape
+    O = out if out is not None else torch.empty((B, Hq, D), dtype=torch.bfloat16, device=Q.device)
+    _check(lib().ef_gqa_decode_static(_ptr(Q, "Q"), _ptr(K, "K"), _ptr(V, "V"), _ptr(O, "O"), B, Hq, Hkv, L, D,
+                                      float(scale), _stream()), "ef_gqa_decode_static")
     return O
 
 

@@ -16,6 +16,8 @@
 // softmax statistics are reduced with warp shuffles.  The kernel moves 2 bytes per 4 flops;
 // tcgen05 would not help it.  All index arithmetic on the merge path is 32-bit: a 64-bit division
 // per element there once cost more than the whole data stream.
+#include <mutex>
+
 #include "host.cuh"
 #include "ptx.cuh"
 
@@ -382,6 +384,56 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
         tmK, tmV, p);
     EF_CUDA_CHECK(cudaGetLastError());
     return EF_OK;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// ef_gqa_decode_static: the same decode attention for callers that cannot allocate
+// ---------------------------------------------------------------------------------------------
+// Scratch for this entry point lives in the library image: every GPU that loads the library
+// holds these bytes until the process exits.  Layout = an ordinary decode workspace (header,
+// one arrival counter per (batch, kv head) unit, partial-state slots of the persistent grid).
+namespace ef {
+namespace decode {
+constexpr int kStaticMaxUnits = 1024;  // B * Hkv accepted by ef_gqa_decode_static
+constexpr size_t kStaticScratchBytes =
+    kHeaderBytes + kStaticMaxUnits * sizeof(uint32_t) + static_cast<size_t>(kMaxGrid) * 2 * kSlotFloats * sizeof(float);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+// On the host, `g_static_scratch` is only a handle for the runtime, not a device address; the
+// address the kernel needs is looked up once per device and cached here.
+static void* g_static_scratch_ptr[64] = {};
+static std::mutex g_static_mu;
+}  // namespace decode
+}  // namespace ef
+
+extern "C" {
+
+size_t ef_gqa_decode_static_max_units(void) { return ef::decode::kStaticMaxUnits; }
+
+ef_status ef_gqa_decode_static(const void* Q, const void* K, const void* V, void* O, int B, int Hq, int Hkv, int L, int D,
+                               float scale, void* stream) {
+    using namespace ef;
+    if (B <= 0 || Hkv <= 0) return EF_ERR_SHAPE;
+    if (static_cast<long long>(B) * Hkv > decode::kStaticMaxUnits) return EF_ERR_WORKSPACE;  // beyond the built-in scratch
+    int dev = -1;
+    EF_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return EF_ERR_UNSUPPORTED;
+    void* ptr = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(decode::g_static_mu);
+        if (!decode::g_static_scratch_ptr[dev]) {
+            // first call on this device (which is current): resolve the array's device address
+            void* p = nullptr;
+            EF_CUDA_CHECK(cudaGetSymbolAddress(&p, decode::g_static_scratch));
+            decode::g_static_scratch_ptr[dev] = p;
+        }
+        ptr = decode::g_static_scratch_ptr[dev];
+    }
+    // The array keeps whatever the previous call left: status word and arrival counters must start at zero.
+    EF_CUDA_CHECK(cudaMemsetAsync(ptr, 0, kHeaderBytes + decode::kStaticMaxUnits * sizeof(uint32_t),
+                                  static_cast<cudaStream_t>(stream)));
+    return ef_gqa_decode(Q, K, V, O, B, Hq, Hkv, L, D, scale, ptr, decode::kStaticScratchBytes, stream);
 }
 
 }  // extern "C"

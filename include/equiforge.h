@@ -99,7 +99,7 @@ size_t ef_gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int L, int D);
  * motion; Section 7.3, QK-normalized MLA).  Score and probability matrices never reach HBM
  * (Section 7.2, "Attention").
  *   Q,K,V [B,H,S,D], gamma_q [D], gamma_k [D] -> O [B,H,S,D].
- * Supported: D == 128, S >= 1. */
+ * Supported: D == 128, S >= 1, scale > 0. */
 ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V,
                          const void* gamma_q, const void* gamma_k, void* O,
                          int B, int H, int S, int D, float eps, float scale, int causal,

@@ -2,10 +2,16 @@
 //
 // Algebra (Table 1, factor motion; Section 7.3, QK-normalized MLA): with rq_i, rk_j the inverse
 // RMS of query row i / key row j,
-//     s_ij = scale * rq_i * rk_j * sum_d q_id (gq_d gk_d) k_jd ,
-// so raw K tiles go TMA -> tensor core untouched, the gamma product is folded into the Q tile
-// once per block, rk_j multiplies the logits column-wise and rq_i * scale * log2(e) row-wise.
-// rk (one float per key) is produced by a small pre-pass kernel; rq is computed in the block.
+//     s_ij = scale * sum_d (rq_i q_id gq_d gk_d) (rk_j k_jd) ,
+// so the gamma product and rq_i are folded into the Q tile once per block (rewritten in shared
+// memory as fp16), scale * log2(e) is folded into the exp2 FMA on the logits, and the key factor is applied
+// once per key by a pre-pass kernel that writes Khat = fp16(k * rk) (read back from L2 by the main
+// kernel; |Khat_d| <= sqrt(128), so fp16's 11-bit mantissa is safe and four times finer than bf16;
+// for the same reason P, which lies in [0, 2^8], is handed to the PV MMA as fp16).  The key factor is NOT applied on the logits inside the block: that needs one
+// shared-memory read per four logits, and shared-memory reads of ordinary warps starve while the
+// tensor core streams Q and K tiles (a 128x128x16 MMA with both operands in shared memory uses the
+// full 128 B/clk; measured: an LDS.128 then takes ~600 cycles).  The softmax loop therefore touches
+// no shared memory at all.
 //
 // Execution form (Figure 4, M2): grid over (batch*head, pair of 128-row Q tiles) = axis m, loop
 // over 128-key K/V tiles = axis p, rolling state <max, sum, value> with the repair
@@ -14,12 +20,12 @@
 // arithmetic because numerator and normaliser use the same one).  Causal: tiles above the
 // diagonal are never visited, only the diagonal tile is masked.
 //
-// Pipeline per block (320 threads): warp 0 = TMA producer (Q once, K/V/rk rings), warp 1 = single
-// thread issuing tcgen05.mma (S_t = Q_t K^T into TMEM, O_t += P_t V with P read from TMEM), warps
-// 2..5 / 6..9 = softmax groups for Q tile 0 / 1 (one thread per row: tcgen05.ld S, exp2, write
-// P as bf16 back into the S columns, rescale O when needed, final O / l).  While one group runs
-// its softmax the tensor core works on the other tile.  Score and probability matrices never
-// leave the SM (Section 7.2).
+// Pipeline per block (320 threads): warp 0 = TMA producer (Q once, K/V rings), warp 1 = single
+// thread issuing tcgen05.mma (S_t = Q_t Khat^T into TMEM, O_t += P_t V with P read from TMEM),
+// warps 2..5 / 6..9 = softmax groups for Q tile 0 / 1 (one thread per row: tcgen05.ld S, packed
+// fp32x2 FMA + exp2, write P as bf16 back into the S columns, rescale O when needed, final
+// O / l).  While one group runs its softmax the tensor core works on the other tile.  Score and
+// probability matrices never leave the SM (Section 7.2).
 #include "host.cuh"
 #include "ptx.cuh"
 
@@ -34,13 +40,11 @@ constexpr int kKVStages = 2;
 constexpr int kThreads = 320;
 constexpr int kSoftmaxThreads = 128;
 constexpr uint32_t kTmemCols = 512;               // S0 | S1 | O0 | O1, 128 fp32 columns each
-constexpr int kRkBytes = kT * 4;
 // shared memory map (offsets from the 1024-aligned base)
 constexpr int kOffQ = 0;                                          // 2 tiles
 constexpr int kOffK = kOffQ + 2 * kTileBytes;                     // kKVStages tiles
 constexpr int kOffV = kOffK + kKVStages * kTileBytes;             // kKVStages tiles
-constexpr int kOffRk = kOffV + kKVStages * kTileBytes;            // [2 groups][2 stages][128 floats]
-constexpr int kOffGamma = kOffRk + 2 * 2 * kRkBytes;              // [128 floats] gq*gk
+constexpr int kOffGamma = kOffV + kKVStages * kTileBytes;         // [128 floats] gq*gk
 constexpr int kOffBars = kOffGamma + kD * 4;
 constexpr int kSmemBytes = 1024 + kOffBars + 512;
 constexpr float kRescaleThreshold = 8.0f;         // log2 units
@@ -48,9 +52,8 @@ constexpr float kRescaleThreshold = 8.0f;         // log2 units
 struct Params {
     const __nv_bfloat16* gamma_q;
     const __nv_bfloat16* gamma_k;
-    const float* rk;      // [BH][s_pad]
     __nv_bfloat16* O;     // [BH][S][128]
-    int BH, S, s_pad, nq, n_pairs, causal;
+    int BH, S, nq, n_pairs, causal;
     float eps, scale_log2;
     uint32_t* status;
 };
@@ -65,30 +68,65 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
                                           uint32_t* status, uint32_t site) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, site)) != 0;
 }
+// Packed fp32x2 arithmetic (sm_100): one instruction works on two adjacent logits.
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 // ---------------------------------------------------------------------------------------------
-// pre-pass: rk[bh][j] = rsqrt(mean_d K[bh][j][d]^2 + eps); 16 threads per key row
+// pre-pass: Khat[row] = fp16(K[row] * rsqrt(mean_d K[row][d]^2 + eps)); 16 threads per key row,
+// one 16-byte piece each, so every load of the grid is in flight at once
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) key_rms_kernel(const __nv_bfloat16* __restrict__ K, float* __restrict__ rk, int BH,
-                                                      int S, int s_pad, float eps) {
-    const long long total = static_cast<long long>(BH) * s_pad;
+__global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16* __restrict__ K,
+                                                            __nv_bfloat16* __restrict__ Khat, long long rows, float eps) {
     const int sub = threadIdx.x & 15;
-    for (long long row = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 4; row < total;
-         row += (static_cast<long long>(gridDim.x) * blockDim.x) >> 4) {
-        const int bh = static_cast<int>(row / s_pad), j = static_cast<int>(row - static_cast<long long>(bh) * s_pad);
-        float ss = 0.f;
-        if (j < S) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(K + (static_cast<size_t>(bh) * S + j) * kD) + sub);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    const long long row = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 4;
+    const bool live = row < rows;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (live) v = __ldg(reinterpret_cast<const uint4*>(K + row * kD) + sub);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float lo[4], hi[4], ss = 0.f;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
-                ss += a * a + b * b;
-            }
-        }
+    for (int i = 0; i < 4; ++i) {
+        lo[i] = __uint_as_float(w[i] << 16);
+        hi[i] = __uint_as_float(w[i] & 0xFFFF0000u);
+        ss += lo[i] * lo[i] + hi[i] * hi[i];
+    }
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (sub == 0) rk[row] = (j < S) ? rsqrtf(ss * (1.f / kD) + eps) : 0.f;
+    for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float rk = rsqrtf(ss * (1.f / kD) + eps);
+    if (live) {
+        uint4 o4;
+        o4.x = pack_f16x2(lo[0] * rk, hi[0] * rk);
+        o4.y = pack_f16x2(lo[1] * rk, hi[1] * rk);
+        o4.z = pack_f16x2(lo[2] * rk, hi[2] * rk);
+        o4.w = pack_f16x2(lo[3] * rk, hi[3] * rk);
+        reinterpret_cast<uint4*>(Khat + row * kD)[sub] = o4;
     }
 }
 
@@ -111,9 +149,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     uint64_t* s_full = bars + 11;            // [2]  MMA -> softmax group t
     uint64_t* p_full = bars + 13;            // [2]  softmax group t -> MMA
     uint64_t* o_done = bars + 15;            // [2]  MMA -> softmax group t (PV finished)
-    uint64_t* rk_full = bars + 17;           // [2 groups][2 stages]
-    uint64_t* rk_empty = bars + 21;          // [2 groups][2 stages]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -136,7 +172,6 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             mbar_init(&v_full[t], 1); mbar_init(&v_empty[t], 1);
             mbar_init(&s_full[t], 1); mbar_init(&p_full[t], 4); mbar_init(&o_done[t], 1);
         }
-        for (int i = 0; i < 4; ++i) { mbar_init(&rk_full[i], 1); mbar_init(&rk_empty[i], 4); }
         *abort_flag = 0u;
         fence_mbar_init();
     }
@@ -167,14 +202,6 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 mbar_expect_tx(&k_full[st], kTileBytes);
                 tma_load_3d(smem + kOffK + st * kTileBytes, &tmK, &k_full[st], 0, j * kT, bh);
                 tma_load_3d(smem + kOffK + st * kTileBytes + kHalfBytes, &tmK, &k_full[st], 64, j * kT, bh);
-                for (int t = 0; t < 2; ++t) {
-                    if (j >= (t == 0 ? n_kv_t0 : n_kv_t1)) continue;
-                    if (!mbar_wait(&rk_empty[t * 2 + st], ph, abort_flag, p.status, 2)) { ok = false; break; }
-                    mbar_expect_tx(&rk_full[t * 2 + st], kRkBytes);
-                    bulk_load_1d(smem + kOffRk + (t * 2 + st) * kRkBytes, p.rk + static_cast<size_t>(bh) * p.s_pad + j * kT,
-                                 kRkBytes, &rk_full[t * 2 + st]);
-                }
-                if (!ok) break;
                 if (!mbar_wait(&v_empty[st], ph, abort_flag, p.status, 3)) break;
                 mbar_expect_tx(&v_full[st], kTileBytes);
                 tma_load_3d(smem + kOffV + st * kTileBytes, &tmV, &v_full[st], 0, j * kT, bh);
@@ -184,24 +211,28 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = make_idesc_bf16(kT, kT, 0, 0);  // A = Q (K-major), B = K (K-major)
-            constexpr uint32_t idesc_pv = make_idesc_bf16(kT, kD, 0, 1);  // A = P (TMEM),    B = V (MN-major)
+            constexpr uint32_t idesc_qk = make_idesc_f16(kT, kT, 0, 0, 0, 0);  // A = Qhat fp16 (K-major), B = Khat fp16 (K-major)
+            constexpr uint32_t idesc_pv = make_idesc_f16(kT, kD, 0, 1, 1, 1);  // A = P bf16 (TMEM),   B = V bf16 (MN-major)
             const uint32_t sQ = smem_u32(smem + kOffQ), sK = smem_u32(smem + kOffK), sV = smem_u32(smem + kOffV);
+            // descriptor words: hi is constant per operand kind, lo = base + compile-time offset
+            constexpr uint32_t hi_kmajor = smem_desc_hi(1024, kSwizzle128B);   // Q and K tiles
+            constexpr uint32_t hi_v = smem_desc_hi(1024, kSwizzle128B);        // V tile (MN-major: LBO in lo word)
+            const uint32_t q_lo[2] = {smem_desc_lo(sQ, 16), smem_desc_lo(sQ + kTileBytes, 16)};
+            const uint32_t k_lo[2] = {smem_desc_lo(sK, 16), smem_desc_lo(sK + kTileBytes, 16)};
+            const uint32_t v_lo[2] = {smem_desc_lo(sV, kHalfBytes), smem_desc_lo(sV + kTileBytes, kHalfBytes)};
             auto issue_qk = [&](int t, int st) {
+                const uint32_t a0 = q_lo[t], b0 = k_lo[st], d = tmem_base + t * kT;
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                    umma_ss(tmem_base + t * kT, make_smem_desc(sQ + t * kTileBytes + off, 16, 1024, kSwizzle128B),
-                            make_smem_desc(sK + st * kTileBytes + off, 16, 1024, kSwizzle128B), idesc_qk, kk != 0 ? 1u : 0u);
+                    const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                    umma_ss_w(d, a0 + off, hi_kmajor, b0 + off, hi_kmajor, idesc_qk, kk != 0 ? 1u : 0u);
                 }
             };
             auto issue_pv = [&](int t, int st, uint32_t accumulate) {
+                const uint32_t b0 = v_lo[st], d = tmem_base + 2 * kT + t * kD, a = tmem_base + t * kT;
 #pragma unroll
-                for (int kk = 0; kk < kT / 16; ++kk) {
-                    umma_ts(tmem_base + 2 * kT + t * kD, tmem_base + t * kT + kk * 8,
-                            make_smem_desc(sV + st * kTileBytes + kk * 2048, kHalfBytes, 1024, kSwizzle128B), idesc_pv,
-                            (accumulate | static_cast<uint32_t>(kk)) != 0 ? 1u : 0u);
-                }
+                for (int kk = 0; kk < kT / 16; ++kk)
+                    umma_ts_w(d, a + kk * 8, b0 + kk * (2048 >> 4), hi_v, idesc_pv, kk != 0 ? 1u : accumulate);
             };
             const int nkv[2] = {n_kv_t0, n_kv_t1};
             bool ok = true;
@@ -258,9 +289,21 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         float rq = 0.f;
         if (ok) ok = warp_wait(q_full, 0u, abort_flag, p.status, 9);
         if (ok) {
-            // rq_i and the in-place rewrite q'_d = bf16(q_d * gq_d * gk_d)
+            // in-place rewrite of this thread's query row: qhat_d = fp16(q_d * rq_i * gq_d * gk_d)
+            // (|q * rq| <= sqrt(128), so fp16 is safe unless the gammas are huge: clamp to its range)
             uint8_t* qrow = smem + kOffQ + t * kTileBytes + r * 128;
             float ss = 0.f;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
+                    ss += a * a + b * b;
+                }
+            }
+            rq = rsqrtf(ss * (1.f / kD) + p.eps);
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
                 uint4* ptr = reinterpret_cast<uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
@@ -269,51 +312,46 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 uint32_t o4[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
-                    ss += a * a + b * b;
-                    o4[i] = pack_bf16x2(a * gprod[c * 8 + 2 * i], b * gprod[c * 8 + 2 * i + 1]);
+                    const float a = __uint_as_float(w[i] << 16) * rq * gprod[c * 8 + 2 * i];
+                    const float b = __uint_as_float(w[i] & 0xFFFF0000u) * rq * gprod[c * 8 + 2 * i + 1];
+                    o4[i] = pack_f16x2(fminf(fmaxf(a, -65504.f), 65504.f), fminf(fmaxf(b, -65504.f), 65504.f));
                 }
                 *ptr = make_uint4(o4[0], o4[1], o4[2], o4[3]);
             }
-            rq = rsqrtf(ss * (1.f / kD) + p.eps) * p.scale_log2;
+            rq = p.scale_log2;   // the logits' only remaining factor: scale * log2(e), the same for every row
             fence_proxy_async_smem();
             mbar_arrive(&q_ready[t]);
         }
+        const uint64_t rq2 = pack_f32x2(__float_as_uint(rq), __float_as_uint(rq));
         float m_ref = -INFINITY, l_sum = 0.f;
         for (int j = 0; j < my_nkv && ok; ++j) {
-            const int st = j & 1;
             if (!warp_wait(&s_full[t], j & 1, abort_flag, p.status, 10)) { ok = false; break; }
-            if (!warp_wait(&rk_full[t * 2 + st], (j >> 1) & 1, abort_flag, p.status, 11)) { ok = false; break; }
             tc_fence_after();
             uint32_t s[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s[c]);
             tmem_wait_ld();
-            const float4* rk4 = reinterpret_cast<const float4*>(smem + kOffRk + (t * 2 + st) * kRkBytes);
             const bool diag = p.causal && (j == qt);
-            const int key0 = j * kT;
-            float umax = -INFINITY;
+            if (diag || (j * kT + kT > p.S)) {  // diagonal tile or ragged last key tile only
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 4; ++c) {
 #pragma unroll
-                for (int i4 = 0; i4 < 8; ++i4) {
-                    const float4 k4 = rk4[c * 8 + i4];
-                    const float kk[4] = {k4.x, k4.y, k4.z, k4.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int col = c * 32 + i4 * 4 + e;
-                        float u = __uint_as_float(s[c][i4 * 4 + e]) * kk[e];
-                        const bool valid = (!diag || col <= r) && (key0 + col < p.S);
-                        u = valid ? u : -INFINITY;
-                        s[c][i4 * 4 + e] = __float_as_uint(u);
-                        umax = fmaxf(umax, u);
+                    for (int i = 0; i < 32; ++i) {
+                        const int col = c * 32 + i;
+                        if (!((!diag || col <= r) && (j * kT + col < p.S))) s[c][i] = 0xFF800000u;  // -inf
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&rk_empty[t * 2 + st]);
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2)
+                    mx[(i >> 1) & 3] = max3(mx[(i >> 1) & 3], __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
+            }
+            const float umax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             // lazy repair of the running maximum
-            const float m_tile = umax * rq;   // rq > 0
+            const float m_tile = umax * rq;   // rq = scale * log2(e) > 0
             float o_scale = 1.f;
             const bool need = m_tile > m_ref + kRescaleThreshold;
             if (need) {
@@ -321,19 +359,26 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 l_sum *= o_scale;
                 m_ref = m_tile;
             }
-            float tile_sum = 0.f;
+            // p = exp2(acc * scale*log2e - m_ref): packed FMA, two exp2, packed row sum (4 independent accumulators)
+            const uint64_t nm2 = pack_f32x2(__float_as_uint(-m_ref), __float_as_uint(-m_ref));
+            uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
             uint32_t pk[64];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(s[c][i]), rq, -m_ref));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(s[c][i + 1]), rq, -m_ref));
-                    tile_sum += p0 + p1;
-                    pk[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
+                for (int i = 0; i < 16; ++i) {
+                    float a, b;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(s[c][2 * i], s[c][2 * i + 1]), rq2, nm2), a, b);
+                    const float p0 = fast_exp2(a), p1 = fast_exp2(b);
+                    acc2[i & 3] = add_f32x2(acc2[i & 3], pack_f32x2(__float_as_uint(p0), __float_as_uint(p1)));
+                    pk[c * 16 + i] = pack_bf16x2(p0, p1);
                 }
             }
-            l_sum += tile_sum;
+            {
+                float a, b;
+                unpack_f32x2(add_f32x2(add_f32x2(acc2[0], acc2[1]), add_f32x2(acc2[2], acc2[3])), a, b);
+                l_sum += a + b;
+            }
             // P (bf16) overwrites the first 64 columns of this thread's own S row
             {
                 uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&pk[0]);
@@ -400,10 +445,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 extern "C" {
 
 size_t ef_qknorm_attn_workspace_bytes(int B, int H, int S, int D) {
-    (void)D;
-    if (B <= 0 || H <= 0 || S <= 0) return 0;
-    const size_t s_pad = (static_cast<size_t>(S) + ef::attn::kT - 1) / ef::attn::kT * ef::attn::kT;
-    return ef::kHeaderBytes + static_cast<size_t>(B) * H * s_pad * sizeof(float);
+    if (B <= 0 || H <= 0 || S <= 0 || D != ef::attn::kD) return 0;
+    return ef::kHeaderBytes + static_cast<size_t>(B) * H * S * D * 2;   // header + Khat (normalised keys, bf16)
 }
 
 ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void* gamma_q, const void* gamma_k, void* O,
@@ -412,7 +455,7 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     using namespace ef;
     if (!Q || !K || !V || !gamma_q || !gamma_k || !O) return EF_ERR_NULL;
     if (B <= 0 || H <= 0 || S <= 0 || D <= 0) return EF_ERR_SHAPE;
-    if (D != attn::kD) return EF_ERR_UNSUPPORTED;
+    if (D != attn::kD || !(scale > 0.f)) return EF_ERR_UNSUPPORTED;
     const long long BH = static_cast<long long>(B) * H;
     const int nq = (S + attn::kT - 1) / attn::kT;
     const int n_pairs = (nq + 1) / 2;
@@ -432,7 +475,9 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     const uint32_t box[3] = {64, attn::kT, 1};
     ef_status st;
     if ((st = encode_tmap_bf16(&tmQ, Q, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
-    if ((st = encode_tmap_bf16(&tmK, K, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    __nv_bfloat16* Khat = reinterpret_cast<__nv_bfloat16*>(w + kHeaderBytes);
+    if ((st = encode_tmap_bf16(&tmK, Khat, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
     if ((st = encode_tmap_bf16(&tmV, V, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
 
     static bool attr_set[64] = {};
@@ -441,25 +486,20 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
                                            attn::kSmemBytes));
         attr_set[di.device] = true;
     }
-    uint8_t* w = static_cast<uint8_t*>(ws);
-    float* rk = reinterpret_cast<float*>(w + kHeaderBytes);
-    const int s_pad = nq * attn::kT;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     {
-        const long long rows = BH * s_pad;
-        long long blocks = (rows * 16 + 255) / 256;
-        const long long cap = static_cast<long long>(di.num_sms) * 16;
-        if (blocks > cap) blocks = cap;
-        attn::key_rms_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(K), rk,
-                                                                          static_cast<int>(BH), S, s_pad, eps);
+        const long long rows = BH * S;
+        const long long blocks = (rows * 16 + 255) / 256;
+        if (blocks > 0x7fffffffLL) return EF_ERR_UNSUPPORTED;
+        attn::key_normalize_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(K), Khat,
+                                                                                rows, eps);
         EF_CUDA_CHECK(cudaGetLastError());
     }
     attn::Params p;
     p.gamma_q = static_cast<const __nv_bfloat16*>(gamma_q);
     p.gamma_k = static_cast<const __nv_bfloat16*>(gamma_k);
-    p.rk = rk;
     p.O = static_cast<__nv_bfloat16*>(O);
-    p.BH = static_cast<int>(BH); p.S = S; p.s_pad = s_pad; p.nq = nq; p.n_pairs = n_pairs; p.causal = causal ? 1 : 0;
+    p.BH = static_cast<int>(BH); p.S = S; p.nq = nq; p.n_pairs = n_pairs; p.causal = causal ? 1 : 0;
     p.eps = eps;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = reinterpret_cast<uint32_t*>(w);

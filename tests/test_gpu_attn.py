@@ -32,6 +32,13 @@ def test_attn_large_eps_and_unit_scale():
     run_parity("qknorm_attn", 6, S=384, eps=0.25, scale=0.02)
 
 
+def test_attn_large_scale_uses_running_max():
+    # logit bound 128 * max|gq gk| * scale * log2(e) > 2^40: the kernel falls back from the a-priori
+    # reference to the running maximum with lazy repair; the softmax is close to one-hot here
+    run_parity("qknorm_attn", 7, S=384, scale=0.5)
+    run_parity("qknorm_attn", 8, S=640, scale=0.35, causal=0)
+
+
 def test_attn_full_config_sampled_heads():
     # full benchmark shape; the oracle's cost is affordable (about 70 GFLOP in fp64)
     r = run_parity("qknorm_attn", 0, size="full", check_repeat=False)

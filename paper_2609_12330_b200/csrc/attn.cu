@@ -107,6 +107,8 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16* __restrict__ K,
                                                             __nv_bfloat16* __restrict__ Khat, long long rows, float eps) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int sub = threadIdx.x & 15;
     const long long row = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 4;
     const bool live = row < rows;
@@ -178,11 +180,13 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         *abort_flag = 0u;
         fence_mbar_init();
     }
+    if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+    pdl_launch_dependents();
+    pdl_wait();  // Khat (previous kernel), gammas, O of earlier calls: no global access above this line
     if (threadIdx.x >= 64 && threadIdx.x < 64 + kD) {
         const int d = threadIdx.x - 64;
         gprod[d] = __bfloat162float(p.gamma_q[d]) * __bfloat162float(p.gamma_k[d]);
     }
-    if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -505,9 +509,8 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
         const long long rows = BH * S;
         const long long blocks = (rows * 16 + 255) / 256;
         if (blocks > 0x7fffffffLL) return EF_ERR_UNSUPPORTED;
-        attn::key_normalize_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(K), Khat,
-                                                                                rows, eps);
-        EF_CUDA_CHECK(cudaGetLastError());
+        EF_CUDA_CHECK(launch_pdl(attn::key_normalize_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s,
+                                 static_cast<const __nv_bfloat16*>(K), Khat, rows, eps));
     }
     attn::Params p;
     p.gamma_q = static_cast<const __nv_bfloat16*>(gamma_q);
@@ -518,8 +521,7 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = reinterpret_cast<uint32_t*>(w);
     const unsigned grid = static_cast<unsigned>(BH * n_pairs);
-    attn::qknorm_attn_kernel<<<grid, attn::kThreads, attn::kSmemBytes, s>>>(tmQ, tmK, tmV, p);
-    EF_CUDA_CHECK(cudaGetLastError());
+    EF_CUDA_CHECK(launch_pdl(attn::qknorm_attn_kernel, dim3(grid), dim3(attn::kThreads), attn::kSmemBytes, s, tmQ, tmK, tmV, p));
     return EF_OK;
 }
 

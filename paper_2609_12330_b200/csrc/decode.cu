@@ -103,7 +103,9 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         *is_last = 0u;
         fence_mbar_init();
     }
+    pdl_launch_dependents();
     __syncthreads();
+    pdl_wait();  // everything below may touch global memory of the previous kernel in the stream
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer warp ------------------------------
@@ -380,9 +382,8 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
     p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
-    decode::gqa_decode_kernel<<<grid, decode::kThreads, decode::kSmemBytes, static_cast<cudaStream_t>(stream)>>>(
-        tmK, tmV, p);
-    EF_CUDA_CHECK(cudaGetLastError());
+    EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
+                             static_cast<cudaStream_t>(stream), tmK, tmV, p));
     return EF_OK;
 }
 

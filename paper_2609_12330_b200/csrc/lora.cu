@@ -67,10 +67,12 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         fence_mbar_init();
     }
     if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // T (previous kernel) and Y of earlier calls: no global access above this line
     const int total_kb = p.k_blocks + p.has_lora;
 
     if (warp == 0) {
@@ -220,10 +222,12 @@ lora_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
         fence_mbar_init();
     }
     if (warp == 1) { tmem_alloc(tmem_slot, kTTmemCols); tmem_relinquish(); }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -418,8 +422,8 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
         tp.M = M; tp.m_pad = pl.m_pad; tp.k_blocks = pl.k_blocks; tp.splits = pl.splits;
         tp.alpha = alpha;
         tp.status = reinterpret_cast<uint32_t*>(w);
-        lora::lora_t_kernel<<<dim3(pl.tiles_m, pl.splits), lora::kTThreads, lora::kTSmemBytes, s>>>(tmX, tmA, tp);
-        EF_CUDA_CHECK(cudaGetLastError());
+        EF_CUDA_CHECK(launch_pdl(lora::lora_t_kernel, dim3(pl.tiles_m, pl.splits), dim3(lora::kTThreads), lora::kTSmemBytes, s,
+                                 tmX, tmA, tp));
     }
     {
         lora::MainParams mp;
@@ -429,8 +433,8 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
         mp.k_blocks = pl.k_blocks; mp.has_lora = 1;
         mp.status = reinterpret_cast<uint32_t*>(w);
         const int grid = di.num_sms < mp.num_tiles ? di.num_sms : mp.num_tiles;
-        lora::lora_main_kernel<<<grid, lora::kThreads, lora::kSmemBytes, s>>>(tmX, tmW, tmT, tmB, mp);
-        EF_CUDA_CHECK(cudaGetLastError());
+        EF_CUDA_CHECK(launch_pdl(lora::lora_main_kernel, dim3(grid), dim3(lora::kThreads), lora::kSmemBytes, s, tmX, tmW, tmT,
+                                 tmB, mp));
     }
     return EF_OK;
 }

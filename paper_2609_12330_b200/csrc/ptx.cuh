@@ -100,6 +100,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 }
 
 // ---------------------------------------------------------------------------------------------
+// programmatic dependent launch: a kernel launched with the programmatic-serialization attribute
+// may start (prologue: barriers, TMEM, tensor-map prefetch) while the previous kernel of the stream
+// drains; pdl_wait() must precede its first global-memory access.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------------------------
 // proxy fences
 // ---------------------------------------------------------------------------------------------
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA / UMMA reads).

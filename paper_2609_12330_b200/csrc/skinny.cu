@@ -29,7 +29,7 @@ constexpr int kWBytes = 2 * kWAtomBytes;          // 16 KiB per weight matrix pe
 constexpr int kXBytes = kMaxM * kBK * 2;          // 2 KiB: [16 rows][64 k] K-major, 128B swizzle
 constexpr int kThreads = 192;                     // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr int kMaxGrid = 256;
-constexpr int kMiscBytes = 512 + kMaxGrid * 4;    // barriers, flags, r_m, slot table
+constexpr int kMiscBytes = 1024 + kMaxGrid * 4;   // barriers, flags, r_m, slot table, row-sum partials
 constexpr int kMaxSmem = 227 * 1024;
 
 struct Params {
@@ -80,6 +80,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
     uint32_t* is_last = tmem_slot + 2;
     float* rinv = reinterpret_cast<float*>(tmem_slot + 4);        // [16]
     int* slot_table = reinterpret_cast<int*>(tmem_slot + 4 + kMaxM);  // [kMaxGrid]
+    float* ssw = reinterpret_cast<float*>(slot_table + kMaxGrid);      // [5 warps][16 rows]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
@@ -93,10 +94,12 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
         fence_mbar_init();
     }
     if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // everything below may touch global memory of the previous kernel in the stream
 
     // The producer starts streaming W right away; everyone else first builds the X operand.
     if (warp == 0) {
@@ -126,33 +129,53 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
         // X operand = bf16(x * gamma) for ALL k blocks, written in the K-major 128B-swizzled tile
         // layout the MMA descriptor expects (row r of a tile: 128 B, 16-byte chunk c stored at
         // chunk c ^ (r & 7)); sum of squares per row for r_m (product fusion: same pass over X).
-        const int w5 = warp - 1;  // 0..4
+        // Thread i of the 160 owns 16-byte column chunk i (+160, ...) of EVERY row: all of a thread's
+        // loads are independent and issued together, so the whole prologue costs one memory latency.
+        const int idx = threadIdx.x - 32;  // 0..159
         const int chunks = p.K >> 3;
-        for (int r = w5; r < kMaxM; r += 5) {
-            float ss = 0.f;
-            for (int c = lane; c < chunks; c += 32) {
-                uint4 xv = make_uint4(0u, 0u, 0u, 0u);
-                if (r < p.M) xv = __ldg(reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(r) * p.K) + c);
-                const uint4 gv = __ldg(reinterpret_cast<const uint4*>(p.gamma) + c);
-                const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
-                const uint32_t gs[4] = {gv.x, gv.y, gv.z, gv.w};
+        float ss[kMaxM];
+#pragma unroll
+        for (int r = 0; r < kMaxM; ++r) ss[r] = 0.f;
+        for (int c = idx; c < chunks; c += 160) {
+            const uint4 gv = __ldg(reinterpret_cast<const uint4*>(p.gamma) + c);
+            uint4 xv[kMaxM];
+#pragma unroll
+            for (int r = 0; r < kMaxM; ++r) {
+                xv[r] = make_uint4(0u, 0u, 0u, 0u);
+                if (r < p.M) xv[r] = __ldg(reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(r) * p.K) + c);
+            }
+            const uint32_t gs[4] = {gv.x, gv.y, gv.z, gv.w};
+            const int kb = c >> 3, cc = c & 7;
+#pragma unroll
+            for (int r = 0; r < kMaxM; ++r) {
+                const uint32_t xs[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w};
                 uint32_t outv[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
                     const float g0 = __uint_as_float(gs[j] << 16), g1 = __uint_as_float(gs[j] & 0xFFFF0000u);
-                    ss += x0 * x0 + x1 * x1;
+                    ss[r] += x0 * x0 + x1 * x1;
                     outv[j] = pack_bf16x2(x0 * g0, x1 * g1);
                 }
-                const int kb = c >> 3, cc = c & 7;
                 *reinterpret_cast<uint4*>(xg + kb * kXBytes + r * 128 + ((cc ^ (r & 7)) << 4)) =
                     make_uint4(outv[0], outv[1], outv[2], outv[3]);
             }
+        }
+        // per-row sum of squares: warp shuffle tree, then the five warp partials in warp order (deterministic)
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            if (lane == 0) rinv[r] = rsqrtf(ss / static_cast<float>(p.K) + p.eps);
+        for (int r = 0; r < kMaxM; ++r) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ss[r] += __shfl_xor_sync(0xffffffffu, ss[r], o);
+            if (lane == 0) ssw[(warp - 1) * kMaxM + r] = ss[r];
         }
         fence_proxy_async_smem();
+        asm volatile("bar.sync 2, 160;" ::: "memory");
+        if (idx < kMaxM) {
+            float tot = 0.f;
+#pragma unroll
+            for (int w = 0; w < 5; ++w) tot += ssw[w * kMaxM + idx];
+            rinv[idx] = rsqrtf(tot / static_cast<float>(p.K) + p.eps);
+        }
     }
     if (NORM && warp != 0) asm volatile("bar.sync 2, 160;" ::: "memory");  // warps 1..5; the producer keeps streaming
 
@@ -352,8 +375,8 @@ ef_status launch(const void* X, const void* gamma, const void* W0, const void* W
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
     p.partials = reinterpret_cast<float*>(w + kHeaderBytes + pl.counters_bytes);
-    skinny_kernel<NW, NORM><<<grid, kThreads, pl.smem_bytes, static_cast<cudaStream_t>(stream)>>>(tmW0, tmW1, tmX, p);
-    EF_CUDA_CHECK(cudaGetLastError());
+    EF_CUDA_CHECK(launch_pdl(skinny_kernel<NW, NORM>, dim3(grid), dim3(kThreads), static_cast<size_t>(pl.smem_bytes),
+                             static_cast<cudaStream_t>(stream), tmW0, tmW1, tmX, p));
     return EF_OK;
 }
 

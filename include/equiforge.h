@@ -59,7 +59,7 @@ typedef enum {
  * the X side; the sum of squares and the K loop form one fused reduction (Table 1, product
  * fusion); W is partitioned along N and K (Table 1, MatMul refinement "NK").
  *   X [M,K], gamma [K], W [K,N] -> Y [M,N].
- * Supported: 1 <= M <= 16, K % 64 == 0, N % 8 == 0. */
+ * Supported: 1 <= M <= 16, K % 64 == 0, K <= 4096, N % 8 == 0. */
 ef_status ef_rmsnorm_matmul(const void* X, const void* gamma, const void* W, void* Y,
                             int M, int K, int N, float eps,
                             void* ws, size_t ws_bytes, void* stream);
@@ -76,6 +76,18 @@ ef_status ef_gated_mlp(const void* X, const void* Wgate, const void* Wup, void* 
                        int M, int K, int N,
                        void* ws, size_t ws_bytes, void* stream);
 size_t ef_gated_mlp_workspace_bytes(int M, int K, int N);
+
+/* ---- Program 2b: RMSNorm fused into the gated MLP (RMSNorm-MLP) ------------------------------
+ * Y = SiLU(Xn @ Wgate) * (Xn @ Wup) with Xn = X * rsqrt(mean(X^2,-1) + eps) * gamma.
+ * Definition: the RMSNorm-MLP workload (Section 7.2): the per-row normalisation factor moves
+ * after each projection, (s (.) X) W == s (.) (X W), and both projections plus the elementwise
+ * product run in ONE kernel with no intermediate in global memory.
+ *   X [M,K], gamma [K], Wgate [K,N], Wup [K,N] -> Y [M,N].
+ * Supported: 1 <= M <= 16, K % 64 == 0, K <= 4096, N % 8 == 0. */
+ef_status ef_rmsnorm_gated_mlp(const void* X, const void* gamma, const void* Wgate, const void* Wup, void* Y,
+                               int M, int K, int N, float eps,
+                               void* ws, size_t ws_bytes, void* stream);
+size_t ef_rmsnorm_gated_mlp_workspace_bytes(int M, int K, int N);
 
 /* ---- Program 3: grouped-query decode attention -------------------------------------------
  * One query token per sequence attends all L cached keys: for query head h and kv head

@@ -65,6 +65,15 @@ def gated_mlp(X, Wgate, Wup):
     return Y
 
 
+def rmsnorm_gated_mlp(X, gamma, Wgate, Wup, eps):
+    X, pX = _d(X); gamma, pg = _d(gamma); Wgate, pG = _d(Wgate); Wup, pU = _d(Wup)
+    M, K = X.shape; N = Wgate.shape[1]
+    assert Wgate.shape == (K, N) and Wup.shape == (K, N) and gamma.shape == (K,)
+    Y = np.empty((M, N), dtype=np.float64)
+    _load().ef_oracle_rmsnorm_gated_mlp(pX, pg, pG, pU, _d(Y)[1], M, K, N, ctypes.c_double(eps))
+    return Y
+
+
 def gqa_decode(Q, K, V, scale):
     Q, pQ = _d(Q); K, pK = _d(K); V, pV = _d(V)
     B, Hq, D = Q.shape; _, Hkv, L, _ = K.shape
@@ -101,6 +110,8 @@ def run(program: str, params: dict, tensors_f64: dict) -> np.ndarray:
         return rmsnorm_matmul(t["X"], t["gamma"], t["W"], p["eps"])
     if program == "gated_mlp":
         return gated_mlp(t["X"], t["Wgate"], t["Wup"])
+    if program == "rmsnorm_gated_mlp":
+        return rmsnorm_gated_mlp(t["X"], t["gamma"], t["Wgate"], t["Wup"], p["eps"])
     if program == "gqa_decode":
         return gqa_decode(t["Q"], t["K"], t["V"], p["scale"])
     if program == "qknorm_attn":

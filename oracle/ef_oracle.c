@@ -92,6 +92,27 @@ void ef_oracle_gated_mlp(const double *X, const double *Wgate, const double *Wup
     }
 }
 
+/* Program 2b (RMSNorm-MLP, Section 7.2): the unfused chain RMSNorm -> two projections -> gate:
+ *   xn_ik = x_ik * r_i * gamma_k;  G = xn @ Wgate;  U = xn @ Wup;  Y = SiLU(G) * U. */
+void ef_oracle_rmsnorm_gated_mlp(const double *X, const double *gamma, const double *Wgate, const double *Wup,
+                                 double *Y, int M, int K, int N, double eps) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < M; ++i) {
+        double *xn = (double *)malloc((size_t)K * sizeof(double));
+        double *g = (double *)malloc((size_t)N * sizeof(double));
+        double *u = (double *)malloc((size_t)N * sizeof(double));
+        const double *x = X + (size_t)i * K;
+        const double r = inv_rms(x, K, eps);
+        for (int k = 0; k < K; ++k) xn[k] = x[k] * r * gamma[k];
+        row_times_matrix(xn, Wgate, g, K, N);
+        row_times_matrix(xn, Wup, u, K, N);
+        for (int n = 0; n < N; ++n) Y[(size_t)i * N + n] = silu(g[n]) * u[n];
+        free(xn);
+        free(g);
+        free(u);
+    }
+}
+
 /* Vanilla attention of ONE query row against n_keys keys (Figure 4, M0):
  *   score = q.k_j (f32-accumulated matmul in the paper; fp64 here), scaled = score*scale,
  *   maximum = max_j scaled, weights = exp(scaled - maximum), normalizer = sum_j weights,

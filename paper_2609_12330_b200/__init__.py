@@ -18,6 +18,7 @@ _lib = None
 EXPORTS = [
     "ef_rmsnorm_matmul", "ef_rmsnorm_matmul_workspace_bytes",
     "ef_gated_mlp", "ef_gated_mlp_workspace_bytes",
+    "ef_rmsnorm_gated_mlp", "ef_rmsnorm_gated_mlp_workspace_bytes",
     "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_static", "ef_gqa_decode_static_max_units",
     "ef_qknorm_attn", "ef_qknorm_attn_workspace_bytes",
     "ef_lora_linear", "ef_lora_linear_workspace_bytes",
@@ -44,6 +45,8 @@ def lib():
         L.ef_rmsnorm_matmul_workspace_bytes.argtypes = [i, i, i]
         L.ef_gated_mlp.argtypes = [vp, vp, vp, vp, i, i, i, vp, sz, vp]
         L.ef_gated_mlp_workspace_bytes.argtypes = [i, i, i]
+        L.ef_rmsnorm_gated_mlp.argtypes = [vp, vp, vp, vp, vp, i, i, i, f, vp, sz, vp]
+        L.ef_rmsnorm_gated_mlp_workspace_bytes.argtypes = [i, i, i]
         L.ef_gqa_decode.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
         L.ef_gqa_decode_workspace_bytes.argtypes = [i, i, i, i, i]
         L.ef_gqa_decode_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp]
@@ -115,6 +118,10 @@ def gated_mlp_workspace_bytes(M, K, N):
     return int(lib().ef_gated_mlp_workspace_bytes(M, K, N))
 
 
+def rmsnorm_gated_mlp_workspace_bytes(M, K, N):
+    return int(lib().ef_rmsnorm_gated_mlp_workspace_bytes(M, K, N))
+
+
 def gqa_decode_workspace_bytes(B, Hq, Hkv, L, D):
     return int(lib().ef_gqa_decode_workspace_bytes(B, Hq, Hkv, L, D))
 
@@ -148,6 +155,18 @@ def gated_mlp(X, Wgate, Wup, ws: Workspace, out=None):
     wp, wb = _ws_args(ws, gated_mlp_workspace_bytes(M, K, N), "ef_gated_mlp")
     _check(lib().ef_gated_mlp(_ptr(X, "X"), _ptr(Wgate, "Wgate"), _ptr(Wup, "Wup"), _ptr(Y, "Y"), M, K, N,
                               wp, wb, _stream()), "ef_gated_mlp")
+    return Y
+
+
+def rmsnorm_gated_mlp(X, gamma, Wgate, Wup, eps, ws: Workspace, out=None):
+    import torch
+
+    M, K = X.shape
+    N = Wgate.shape[1]
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    wp, wb = _ws_args(ws, rmsnorm_gated_mlp_workspace_bytes(M, K, N), "ef_rmsnorm_gated_mlp")
+    _check(lib().ef_rmsnorm_gated_mlp(_ptr(X, "X"), _ptr(gamma, "gamma"), _ptr(Wgate, "Wgate"), _ptr(Wup, "Wup"),
+                                      _ptr(Y, "Y"), M, K, N, float(eps), wp, wb, _stream()), "ef_rmsnorm_gated_mlp")
     return Y
 
 
@@ -208,6 +227,8 @@ def workspace_bytes(program: str, p: dict) -> int:
         return rmsnorm_matmul_workspace_bytes(p["M"], p["K"], p["N"])
     if program == "gated_mlp":
         return gated_mlp_workspace_bytes(p["M"], p["K"], p["N"])
+    if program == "rmsnorm_gated_mlp":
+        return rmsnorm_gated_mlp_workspace_bytes(p["M"], p["K"], p["N"])
     if program == "gqa_decode":
         return gqa_decode_workspace_bytes(p["B"], p["Hq"], p["Hkv"], p["L"], p["D"])
     if program == "qknorm_attn":
@@ -223,6 +244,8 @@ def run(program: str, p: dict, t: dict, ws: Workspace, out=None):
         return rmsnorm_matmul(t["X"], t["gamma"], t["W"], p["eps"], ws, out)
     if program == "gated_mlp":
         return gated_mlp(t["X"], t["Wgate"], t["Wup"], ws, out)
+    if program == "rmsnorm_gated_mlp":
+        return rmsnorm_gated_mlp(t["X"], t["gamma"], t["Wgate"], t["Wup"], p["eps"], ws, out)
     if program == "gqa_decode":
         return gqa_decode(t["Q"], t["K"], t["V"], p["scale"], ws, out)
     if program == "qknorm_attn":

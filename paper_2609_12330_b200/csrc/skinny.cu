@@ -14,7 +14,8 @@
 // axis, deterministic) and only then applies the pointwise epilogue -- SiLU(gate)*up is nonlinear,
 // so it cannot be applied to partial sums; the RMSNorm row factor r_m is invariant along K and is
 // applied at the same place (Table 1, factor motion), while gamma varies along K and is folded
-// into the X operand when the block builds it.
+// into the X operand when the block builds it.  The same kernel with both options on is the
+// RMSNorm-MLP program: Y = SiLU(r (X gamma) Wg) * (r (X gamma) Wu) in one launch.
 #include "host.cuh"
 #include "ptx.cuh"
 
@@ -83,6 +84,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
     float* ssw = reinterpret_cast<float*>(slot_table + kMaxGrid);      // [5 warps][16 rows]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool split = NORM && p.M <= 8;   // X operand as hi/lo row pairs (see the prologue)
     const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
     const int it_end = range_begin(blockIdx.x + 1, p.base, p.rem);
 
@@ -146,19 +148,44 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
             }
             const uint32_t gs[4] = {gv.x, gv.y, gv.z, gv.w};
             const int kb = c >> 3, cc = c & 7;
+            if (split) {
+                // M <= 8: rows 0..7 hold hi = bf16(x*gamma), rows 8..15 hold lo = bf16(x*gamma - hi); the MMA
+                // produces both partial results at no extra cost and the epilogue adds them, so the X
+                // operand effectively carries 16 mantissa bits (x and gamma are bf16: the product has 16).
 #pragma unroll
-            for (int r = 0; r < kMaxM; ++r) {
-                const uint32_t xs[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w};
-                uint32_t outv[4];
+                for (int r = 0; r < 8; ++r) {
+                    const uint32_t xs[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w};
+                    uint32_t hi4[4], lo4[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
-                    const float g0 = __uint_as_float(gs[j] << 16), g1 = __uint_as_float(gs[j] & 0xFFFF0000u);
-                    ss[r] += x0 * x0 + x1 * x1;
-                    outv[j] = pack_bf16x2(x0 * g0, x1 * g1);
+                    for (int j = 0; j < 4; ++j) {
+                        const float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
+                        const float g0 = __uint_as_float(gs[j] << 16), g1 = __uint_as_float(gs[j] & 0xFFFF0000u);
+                        ss[r] += x0 * x0 + x1 * x1;
+                        const float v0 = x0 * g0, v1 = x1 * g1;
+                        hi4[j] = pack_bf16x2(v0, v1);
+                        const float h0 = __uint_as_float(hi4[j] << 16), h1 = __uint_as_float(hi4[j] & 0xFFFF0000u);
+                        lo4[j] = pack_bf16x2(v0 - h0, v1 - h1);
+                    }
+                    *reinterpret_cast<uint4*>(xg + kb * kXBytes + r * 128 + ((cc ^ (r & 7)) << 4)) =
+                        make_uint4(hi4[0], hi4[1], hi4[2], hi4[3]);
+                    *reinterpret_cast<uint4*>(xg + kb * kXBytes + (r + 8) * 128 + ((cc ^ (r & 7)) << 4)) =
+                        make_uint4(lo4[0], lo4[1], lo4[2], lo4[3]);
                 }
-                *reinterpret_cast<uint4*>(xg + kb * kXBytes + r * 128 + ((cc ^ (r & 7)) << 4)) =
-                    make_uint4(outv[0], outv[1], outv[2], outv[3]);
+            } else {
+#pragma unroll
+                for (int r = 0; r < kMaxM; ++r) {
+                    const uint32_t xs[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w};
+                    uint32_t outv[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
+                        const float g0 = __uint_as_float(gs[j] << 16), g1 = __uint_as_float(gs[j] & 0xFFFF0000u);
+                        ss[r] += x0 * x0 + x1 * x1;
+                        outv[j] = pack_bf16x2(x0 * g0, x1 * g1);
+                    }
+                    *reinterpret_cast<uint4*>(xg + kb * kXBytes + r * 128 + ((cc ^ (r & 7)) << 4)) =
+                        make_uint4(outv[0], outv[1], outv[2], outv[3]);
+                }
             }
         }
         // per-row sum of squares: warp shuffle tree, then the five warp partials in warp order (deterministic)
@@ -280,10 +307,16 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
 #pragma unroll
                 for (int m = 0; m < kMaxM; ++m) {
                     if (m < p.M) {
+                        // r_m is invariant along K: it scales each finished projection (factor motion)
+                        const float r = NORM ? rinv[m] : 1.f;
+                        float a0 = __uint_as_float(v[0][m]), a1 = __uint_as_float(v[NW - 1][m]);
+                        if (split) {  // hi + lo halves of the X operand (m < 8 here)
+                            a0 += __uint_as_float(v[0][(m + 8) & 15]);
+                            a1 += __uint_as_float(v[NW - 1][(m + 8) & 15]);
+                        }
                         float y;
-                        if (NW == 2) y = silu(__uint_as_float(v[0][m])) * __uint_as_float(v[NW - 1][m]);
-                        else y = __uint_as_float(v[0][m]);
-                        if (NORM) y *= rinv[m];
+                        if (NW == 2) y = silu(a0 * r) * (a1 * r);
+                        else y = a0 * r;
                         p.Y[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
                     }
                 }
@@ -393,6 +426,16 @@ size_t ef_rmsnorm_matmul_workspace_bytes(int M, int K, int N) {
 ef_status ef_rmsnorm_matmul(const void* X, const void* gamma, const void* W, void* Y, int M, int K, int N, float eps,
                             void* ws, size_t ws_bytes, void* stream) {
     return ef::skinny::launch<1, true>(X, gamma, W, nullptr, Y, M, K, N, eps, ws, ws_bytes, stream);
+}
+
+size_t ef_rmsnorm_gated_mlp_workspace_bytes(int M, int K, int N) {
+    ef::skinny::Plan pl;
+    if (M <= 0 || K <= 0 || N <= 0 || K % ef::skinny::kBK != 0 || !ef::skinny::make_plan(2, true, K, N, &pl)) return 0;
+    return pl.total;
+}
+ef_status ef_rmsnorm_gated_mlp(const void* X, const void* gamma, const void* Wgate, const void* Wup, void* Y, int M, int K,
+                               int N, float eps, void* ws, size_t ws_bytes, void* stream) {
+    return ef::skinny::launch<2, true>(X, gamma, Wgate, Wup, Y, M, K, N, eps, ws, ws_bytes, stream);
 }
 
 size_t ef_gated_mlp_workspace_bytes(int M, int K, int N) {

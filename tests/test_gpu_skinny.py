@@ -60,3 +60,19 @@ def test_rmsnorm_matmul_large_eps_and_zero_row():
 def test_rmsnorm_matmul_full_config():
     r = run_parity("rmsnorm_matmul", 0, size="full")
     assert r["rel_l2"] < 5e-3
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_rmsnorm_gated_mlp_small_ragged(seed):
+    r = run_parity("rmsnorm_gated_mlp", seed)     # M=5, K=192, N=200
+    assert r["rel_l2"] < 5e-3
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 64, 8), (16, 4096, 264), (9, 1024, 1000)])
+def test_rmsnorm_gated_mlp_shapes(M, K, N):
+    run_parity("rmsnorm_gated_mlp", 3, M=M, K=K, N=N)
+
+
+def test_rmsnorm_gated_mlp_full_config():
+    r = run_parity("rmsnorm_gated_mlp", 0, size="full")   # batch 8, 4096 -> 11008
+    assert r["rel_l2"] < 5e-3

@@ -156,6 +156,49 @@ def test_gated_mlp_column_combination_and_split_k():
 
 
 # ----------------------------------------------------------------------------
+# Program 2b: RMSNorm fused into the gated MLP
+# ----------------------------------------------------------------------------
+def test_rmsnorm_gated_mlp_unit_rms_rows_library_case():
+    # rows of +-1 have mean square 1: at eps == 0 the normalisation is the identity and
+    # Y == G*expit(G)*U with G = (X*gamma)@Wg, U = (X*gamma)@Wu (numpy + scipy only)
+    M, K, N = 3, 8, 5
+    X = RNG.choice([-1.0, 1.0], size=(M, K)); gamma = RNG.standard_normal(K)
+    Wg = RNG.standard_normal((K, N)); Wu = RNG.standard_normal((K, N))
+    G, U = (X * gamma) @ Wg, (X * gamma) @ Wu
+    np.testing.assert_allclose(oracle.rmsnorm_gated_mlp(X, gamma, Wg, Wu, 0.0), G * expit(G) * U, **TOL)
+
+
+def test_rmsnorm_gated_mlp_factor_motion_after_each_projection():
+    # Section 7.2: (s (.) X) W == s (.) (X W): the row factor applied after BOTH projections
+    M, K, N = 4, 6, 7
+    X = RNG.standard_normal((M, K)); gamma = 1.0 + 0.1 * RNG.standard_normal(K)
+    Wg = RNG.standard_normal((K, N)); Wu = RNG.standard_normal((K, N)); eps = 1e-2
+    r = 1.0 / np.sqrt((X ** 2).mean(1, keepdims=True) + eps)
+    G, U = r * ((X * gamma) @ Wg), r * ((X * gamma) @ Wu)
+    y = oracle.rmsnorm_gated_mlp(X, gamma, Wg, Wu, eps)
+    np.testing.assert_allclose(y, G * expit(G) * U, **TOL)
+    # ties to the pinned single-projection oracle: the two normalised projections, then the gate
+    g1 = oracle.rmsnorm_matmul(X, gamma, Wg, eps); u1 = oracle.rmsnorm_matmul(X, gamma, Wu, eps)
+    np.testing.assert_allclose(y, g1 * expit(g1) * u1, **TOL)
+    # the row factor must NOT be applied once to the product (SiLU is not homogeneous)
+    G0, U0 = (X * gamma) @ Wg, (X * gamma) @ Wu
+    assert not np.allclose(y, r * (G0 * expit(G0) * U0))
+
+
+def test_rmsnorm_gated_mlp_invariants():
+    K, N = 8, 4
+    X = RNG.standard_normal((2, K)); X[1] = 0.0
+    gamma = RNG.standard_normal(K); Wg = RNG.standard_normal((K, N)); Wu = RNG.standard_normal((K, N))
+    y = oracle.rmsnorm_gated_mlp(X, gamma, Wg, Wu, 1e-6)
+    assert np.all(np.isfinite(y)) and np.all(y[1] == 0.0)          # zero row
+    Xs = X.copy(); Xs[0] *= 13.0                                     # eps == 0: row scale invariance
+    np.testing.assert_allclose(oracle.rmsnorm_gated_mlp(Xs[:1], gamma, Wg, Wu, 0.0),
+                               oracle.rmsnorm_gated_mlp(X[:1], gamma, Wg, Wu, 0.0), **TOL)
+    assert not np.allclose(oracle.rmsnorm_gated_mlp(X[:1], gamma, Wu, Wg, 0.0),
+                           oracle.rmsnorm_gated_mlp(X[:1], gamma, Wg, Wu, 0.0))  # which projection is gated
+
+
+# ----------------------------------------------------------------------------
 # Program 3: GQA decode attention (M0 of Figure 4, one query row)
 # ----------------------------------------------------------------------------
 def _m2_rolling(q, K, V, scale, tile_bounds):

@@ -21,7 +21,9 @@ from __future__ import annotations
 import numpy as np
 
 PROGRAMS = ("rmsnorm_matmul", "gated_mlp", "gqa_decode", "qknorm_attn", "lora_linear")
-_PROGRAM_ID = {name: i for i, name in enumerate(PROGRAMS)}
+# programs beyond the five benchmark configurations (the "next" rows of the scope table)
+EXTRA_PROGRAMS = ("rmsnorm_gated_mlp",)
+_PROGRAM_ID = {name: i for i, name in enumerate(PROGRAMS + EXTRA_PROGRAMS)}
 
 
 # ----------------------------------------------------------------------------
@@ -82,6 +84,10 @@ SHAPES = {
         "full": dict(M=16, K=4096, N=11008),
         "small": dict(M=11, K=320, N=200),
     },
+    "rmsnorm_gated_mlp": {  # RMSNorm-MLP at batch 8 (Section 7.2), Llama-2-7B MLP shape
+        "full": dict(M=8, K=4096, N=11008, eps=1e-6),
+        "small": dict(M=5, K=192, N=200, eps=1e-6),
+    },
     "gqa_decode": {
         "full": dict(B=8, Hq=32, Hkv=8, L=4096, D=128, scale=1.0 / np.sqrt(128.0)),
         "small": dict(B=2, Hq=8, Hkv=2, L=333, D=128, scale=1.0 / np.sqrt(128.0)),
@@ -116,6 +122,14 @@ def make_inputs(program: str, seed: int = 0, size: str = "full", **overrides):
             "X": g(0, (M, K), 0.0, 1.0),
             "Wgate": g(1, (K, N), 0.0, 1.0 / np.sqrt(K)),
             "Wup": g(2, (K, N), 0.0, 1.0 / np.sqrt(K)),
+        }
+    elif program == "rmsnorm_gated_mlp":
+        M, K, N = p["M"], p["K"], p["N"]
+        t = {
+            "X": g(0, (M, K), 0.0, 1.0),
+            "gamma": g(1, (K,), 1.0, 0.1),
+            "Wgate": g(2, (K, N), 0.0, 1.0 / np.sqrt(K)),
+            "Wup": g(3, (K, N), 0.0, 1.0 / np.sqrt(K)),
         }
     elif program == "gqa_decode":
         B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
@@ -154,6 +168,9 @@ def algorithmic_work(program: str, p: dict) -> dict:
     if program == "gated_mlp":
         M, K, N = p["M"], p["K"], p["N"]
         return dict(flops=4 * M * K * N, bytes=2 * (2 * K * N + M * K + M * N))
+    if program == "rmsnorm_gated_mlp":
+        M, K, N = p["M"], p["K"], p["N"]
+        return dict(flops=4 * M * K * N, bytes=2 * (2 * K * N + M * K + K + M * N))
     if program == "gqa_decode":
         B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
         return dict(flops=4 * B * Hq * L * D, bytes=2 * (2 * B * Hkv * L * D + 2 * B * Hq * D))

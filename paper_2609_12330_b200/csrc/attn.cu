@@ -13,7 +13,9 @@
 // full 128 B/clk; measured: an LDS.128 then takes ~600 cycles).  The softmax loop therefore touches
 // no shared memory at all.
 //
-// Execution form (Figure 4, M2): grid over (batch*head, pair of 128-row Q tiles) = axis m, loop
+// Execution form (Figure 4, M2): work items (batch*head, pair of 128-row Q tiles) = axis m, pulled
+// heaviest-first from a global counter by one persistent block per SM (the next item's Q tiles
+// are fetched while the current item drains); loop
 // over 128-key K/V tiles = axis p, rolling state <max, sum, value> with the repair
 // h(c,s,s') = c * exp(s - s').  The repair is applied lazily: the accumulated value is rescaled
 // only when the running maximum grows by more than 2^8 (any reference maximum is exact in real
@@ -38,17 +40,18 @@ constexpr int kD = 128;
 constexpr int kT = 128;                           // tile edge (queries and keys)
 constexpr int kHalfBytes = kT * 128;              // [128 rows][64 d] bf16, 128B swizzle
 constexpr int kTileBytes = 2 * kHalfBytes;        // 32 KiB
-constexpr int kKVStages = 2;
+constexpr int kKVSlots = 5;                        // one ring for K and V tiles: K_j, V_j, K_j+1, V_j+1, K_j+2
 constexpr int kThreads = 320;
 constexpr int kSoftmaxThreads = 128;
 constexpr uint32_t kTmemCols = 512;               // S0 | S1 | O0 | O1, 128 fp32 columns each
 // shared memory map (offsets from the 1024-aligned base)
 constexpr int kOffQ = 0;                                          // 2 tiles
-constexpr int kOffK = kOffQ + 2 * kTileBytes;                     // kKVStages tiles
-constexpr int kOffV = kOffK + kKVStages * kTileBytes;             // kKVStages tiles
-constexpr int kOffGamma = kOffV + kKVStages * kTileBytes;         // [128 floats] gq*gk
+constexpr int kOffKV = kOffQ + 2 * kTileBytes;                    // kKVSlots tiles
+constexpr int kOffGamma = kOffKV + kKVSlots * kTileBytes;         // [128 floats] gq*gk
 constexpr int kOffBars = kOffGamma + kD * 4;
 constexpr int kSmemBytes = 1024 + kOffBars + 512;
+constexpr int kWorkCounterWord = 16;               // uint32 index into the workspace header
+constexpr int kDoneCounterWord = 17;
 constexpr float kRescaleThreshold = 8.0f;         // log2 units
 constexpr float kFixedRefLimit = 40.0f;           // log2 units: use the a-priori logit bound as softmax reference
 
@@ -58,7 +61,9 @@ struct Params {
     __nv_bfloat16* O;     // [BH][S][128]
     int BH, S, nq, n_pairs, causal;
     float eps, scale_log2;
+    int total_items;
     uint32_t* status;
+    uint32_t* header;   // workspace header: work counter / done counter for the persistent grid
 };
 
 __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
@@ -136,8 +141,27 @@ __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16*
 }
 
 // ---------------------------------------------------------------------------------------------
-// main kernel
+// main kernel (persistent: one block per SM pulls work items from a global counter)
 // ---------------------------------------------------------------------------------------------
+// Work item = (batch*head, pair of Q tiles); item index order is heaviest pair first, so greedy
+// pulling is longest-processing-time-first scheduling.
+struct Item {
+    int bh, qt0, n_kv, nkv0, nkv1;
+};
+__device__ __forceinline__ Item item_geom(const Params& p, int item) {
+    Item g;
+    const int pair = p.n_pairs - 1 - item / p.BH;
+    g.bh = item - (item / p.BH) * p.BH;
+    g.qt0 = 2 * pair;
+    const int qt1 = g.qt0 + 1;
+    const bool has_q1 = qt1 < p.nq;
+    const int q_last = has_q1 ? qt1 : g.qt0;
+    g.n_kv = p.causal ? (q_last + 1) : p.nq;                       // key tiles the pair visits
+    g.nkv0 = p.causal ? (g.qt0 + 1) : p.nq;                        // ... and each of its two Q tiles
+    g.nkv1 = has_q1 ? (p.causal ? (qt1 + 1) : p.nq) : 0;
+    return g;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const Params p) {
@@ -145,38 +169,31 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float* gprod = reinterpret_cast<float*>(smem + kOffGamma);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kOffBars);
-    uint64_t* q_full = bars;                 // [1]
-    uint64_t* q_ready = bars + 1;            // [2]  softmax group -> MMA (Q tile rewritten)
-    uint64_t* k_full = bars + 3;             // [2]
-    uint64_t* k_empty = bars + 5;            // [2]
-    uint64_t* v_full = bars + 7;             // [2]
-    uint64_t* v_empty = bars + 9;            // [2]
-    uint64_t* s_full = bars + 11;            // [2]  MMA -> softmax group t
-    uint64_t* p_full = bars + 13;            // [2]  softmax group t -> MMA
-    uint64_t* o_done = bars + 15;            // [2]  MMA -> softmax group t (PV finished)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+    uint64_t* q_full = bars;                 // [2]  TMA -> softmax group t (raw Q tile t of the item landed)
+    uint64_t* q_empty = bars + 2;            // [2]  MMA -> TMA (last QK^T of tile t done: Q tile t may be overwritten)
+    uint64_t* q_ready = bars + 4;            // [2]  softmax group t -> MMA (Q tile t rewritten)
+    uint64_t* kv_full = bars + 6;            // [5]  K/V ring: load number n (K of key tile c: n = 2c, V: n = 2c+1)
+    uint64_t* kv_empty = bars + 11;          // [5]        lives in slot n % 5, phase (n / 5) & 1
+    uint64_t* s_full = bars + 16;            // [2]  MMA -> softmax group t
+    uint64_t* p_full = bars + 18;            // [2]  softmax group t -> MMA
+    uint64_t* o_done = bars + 20;            // [2]  MMA -> softmax group t (PV finished)
+    uint64_t* o_free = bars + 22;            // [2]  softmax group t -> MMA (O_t read out: may be overwritten)
+    uint64_t* item_full = bars + 24;         // [2]  TMA -> everyone (work item published)
+    uint64_t* item_empty = bars + 26;        // [2]  everyone -> TMA (item slot read)
+    int* item_ring = reinterpret_cast<int*>(bars + 28);   // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 29);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // heaviest (latest) Q tile pairs first: blocks are dispatched in index order
-    const int pair = p.n_pairs - 1 - static_cast<int>(blockIdx.x / p.BH);
-    const int bh = static_cast<int>(blockIdx.x % p.BH);
-    const int qt0 = 2 * pair, qt1 = 2 * pair + 1;
-    const bool has_q1 = qt1 < p.nq;
-    const int q_last = has_q1 ? qt1 : qt0;
-    const int n_kv = p.causal ? (q_last + 1) : p.nq;
-    // number of key tiles each Q tile visits
-    const int n_kv_t0 = p.causal ? (qt0 + 1) : p.nq;
-    const int n_kv_t1 = has_q1 ? (p.causal ? (qt1 + 1) : p.nq) : 0;
 
     if (threadIdx.x == 0) {
-        mbar_init(q_full, 1);
         for (int t = 0; t < 2; ++t) {
+            mbar_init(&q_full[t], 1); mbar_init(&q_empty[t], 1);
             mbar_init(&q_ready[t], kSoftmaxThreads);
-            mbar_init(&k_full[t], 1); mbar_init(&k_empty[t], 1);
-            mbar_init(&v_full[t], 1); mbar_init(&v_empty[t], 1);
-            mbar_init(&s_full[t], 1); mbar_init(&p_full[t], 4); mbar_init(&o_done[t], 1);
+            mbar_init(&s_full[t], 1); mbar_init(&p_full[t], 4); mbar_init(&o_done[t], 1); mbar_init(&o_free[t], 4);
+            mbar_init(&item_full[t], 1); mbar_init(&item_empty[t], 9);   // MMA thread + 8 softmax warps
         }
+        for (int i = 0; i < kKVSlots; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); }
         *abort_flag = 0u;
         fence_mbar_init();
     }
@@ -193,26 +210,59 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------ TMA producer ------------------------------
+        // ------------------------------ TMA producer + work fetch ------------------------------
         if (lane == 0) {
             tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-            mbar_expect_tx(q_full, 2 * kTileBytes);
-            for (int t = 0; t < 2; ++t) {   // rows beyond S are out of bounds -> zero fill
-                tma_load_3d(smem + kOffQ + t * kTileBytes, &tmQ, q_full, 0, (qt0 + t) * kT, bh);
-                tma_load_3d(smem + kOffQ + t * kTileBytes + kHalfBytes, &tmQ, q_full, 64, (qt0 + t) * kT, bh);
-            }
+            uint32_t kv_count = 0;   // key tiles loaded so far (stage / phase of the K and V rings)
+            uint32_t n_items = 0;
+            uint32_t item = atomicAdd(&p.header[kWorkCounterWord], 1u);
             bool ok = true;
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const int st = j & 1;
-                const uint32_t ph = ((j >> 1) & 1) ^ 1u;
-                if (!mbar_wait(&k_empty[st], ph, abort_flag, p.status, 1)) break;
-                mbar_expect_tx(&k_full[st], kTileBytes);
-                tma_load_3d(smem + kOffK + st * kTileBytes, &tmK, &k_full[st], 0, j * kT, bh);
-                tma_load_3d(smem + kOffK + st * kTileBytes + kHalfBytes, &tmK, &k_full[st], 64, j * kT, bh);
-                if (!mbar_wait(&v_empty[st], ph, abort_flag, p.status, 3)) break;
-                mbar_expect_tx(&v_full[st], kTileBytes);
-                tma_load_3d(smem + kOffV + st * kTileBytes, &tmV, &v_full[st], 0, j * kT, bh);
-                tma_load_3d(smem + kOffV + st * kTileBytes + kHalfBytes, &tmV, &v_full[st], 64, j * kT, bh);
+            while (ok) {
+                const int slot = n_items & 1;
+                if (!mbar_wait(&item_empty[slot], ((n_items >> 1) & 1) ^ 1u, abort_flag, p.status, 1)) break;
+                const bool valid = item < static_cast<uint32_t>(p.total_items);
+                item_ring[slot] = valid ? static_cast<int>(item) : -1;
+                mbar_arrive(&item_full[slot]);
+                if (!valid) break;
+                const uint32_t next = atomicAdd(&p.header[kWorkCounterWord], 1u);   // latency hides behind the copies
+                const Item g = item_geom(p, static_cast<int>(item));
+                // Q tile t of the new item goes in as soon as the previous item's last QK^T of tile t is done
+                // (tile 0 finishes one key tile earlier than tile 1 under the causal mask), so the load is
+                // hidden behind the previous item's tail.  Order: Q0, K(0), Q1, V(0), then the remaining K/V.
+                auto load_q = [&](int t) -> bool {
+                    if (n_items > 0 && !mbar_wait(&q_empty[t], (n_items - 1) & 1, abort_flag, p.status, 2)) return false;
+                    mbar_expect_tx(&q_full[t], kTileBytes);   // rows beyond S are out of bounds -> zero fill
+                    tma_load_3d(smem + kOffQ + t * kTileBytes, &tmQ, &q_full[t], 0, (g.qt0 + t) * kT, g.bh);
+                    tma_load_3d(smem + kOffQ + t * kTileBytes + kHalfBytes, &tmQ, &q_full[t], 64, (g.qt0 + t) * kT, g.bh);
+                    return true;
+                };
+                if (!load_q(0)) break;
+                for (int j = 0; j < g.n_kv; ++j, ++kv_count) {
+                    {
+                        const uint32_t n = 2 * kv_count, sl = n % kKVSlots;
+                        if (!mbar_wait(&kv_empty[sl], ((n / kKVSlots) & 1) ^ 1u, abort_flag, p.status, 3)) { ok = false; break; }
+                        mbar_expect_tx(&kv_full[sl], kTileBytes);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmK, &kv_full[sl], 0, j * kT, g.bh);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmK, &kv_full[sl], 64, j * kT, g.bh);
+                    }
+                    if (j == 0 && !load_q(1)) { ok = false; break; }
+                    {
+                        const uint32_t n = 2 * kv_count + 1, sl = n % kKVSlots;
+                        if (!mbar_wait(&kv_empty[sl], ((n / kKVSlots) & 1) ^ 1u, abort_flag, p.status, 3)) { ok = false; break; }
+                        mbar_expect_tx(&kv_full[sl], kTileBytes);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmV, &kv_full[sl], 0, j * kT, g.bh);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmV, &kv_full[sl], 64, j * kT, g.bh);
+                    }
+                }
+                item = next;
+                ++n_items;
+            }
+            // The block that stops fetching last re-arms the work counter for the next call.
+            __threadfence();
+            const uint32_t prev = atomicAdd(&p.header[kDoneCounterWord], 1u);
+            if (prev == gridDim.x - 1) {
+                p.header[kWorkCounterWord] = 0u;
+                p.header[kDoneCounterWord] = 0u;
             }
         }
     } else if (warp == 1) {
@@ -220,65 +270,92 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (lane == 0) {
             constexpr uint32_t idesc_qk = make_idesc_f16(kT, kT, 0, 0, 0, 0);  // A = Qhat fp16 (K-major), B = Khat fp16 (K-major)
             constexpr uint32_t idesc_pv = make_idesc_f16(kT, kD, 0, 1, 1, 1);  // A = P bf16 (TMEM),   B = V bf16 (MN-major)
-            const uint32_t sQ = smem_u32(smem + kOffQ), sK = smem_u32(smem + kOffK), sV = smem_u32(smem + kOffV);
+            const uint32_t sQ = smem_u32(smem + kOffQ), sKV = smem_u32(smem + kOffKV);
             // descriptor words: hi is constant per operand kind, lo = base + compile-time offset
             constexpr uint32_t hi_kmajor = smem_desc_hi(1024, kSwizzle128B);   // Q and K tiles
             constexpr uint32_t hi_v = smem_desc_hi(1024, kSwizzle128B);        // V tile (MN-major: LBO in lo word)
             const uint32_t q_lo[2] = {smem_desc_lo(sQ, 16), smem_desc_lo(sQ + kTileBytes, 16)};
-            const uint32_t k_lo[2] = {smem_desc_lo(sK, 16), smem_desc_lo(sK + kTileBytes, 16)};
-            const uint32_t v_lo[2] = {smem_desc_lo(sV, kHalfBytes), smem_desc_lo(sV + kTileBytes, kHalfBytes)};
-            auto issue_qk = [&](int t, int st) {
-                const uint32_t a0 = q_lo[t], b0 = k_lo[st], d = tmem_base + t * kT;
+            auto issue_qk = [&](int t, uint32_t slot) {
+                const uint32_t a0 = q_lo[t], b0 = smem_desc_lo(sKV + slot * kTileBytes, 16), d = tmem_base + t * kT;
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
                     umma_ss_w(d, a0 + off, hi_kmajor, b0 + off, hi_kmajor, idesc_qk, kk != 0 ? 1u : 0u);
                 }
             };
-            auto issue_pv = [&](int t, int st, uint32_t accumulate) {
-                const uint32_t b0 = v_lo[st], d = tmem_base + 2 * kT + t * kD, a = tmem_base + t * kT;
+            auto issue_pv = [&](int t, uint32_t slot, uint32_t accumulate) {
+                const uint32_t b0 = smem_desc_lo(sKV + slot * kTileBytes, kHalfBytes), d = tmem_base + 2 * kT + t * kD, a = tmem_base + t * kT;
 #pragma unroll
                 for (int kk = 0; kk < kT / 16; ++kk)
                     umma_ts_w(d, a + kk * 8, b0 + kk * (2048 >> 4), hi_v, idesc_pv, kk != 0 ? 1u : accumulate);
             };
-            const int nkv[2] = {n_kv_t0, n_kv_t1};
+            uint32_t kv_use = 0;          // key tiles consumed by earlier items
+            uint32_t n_items = 0;
+            uint32_t cp[2] = {0u, 0u};    // p_full completions consumed per tile
             bool ok = true;
-            for (int t = 0; t < 2 && ok; ++t)
-                if (nkv[t] > 0) ok = mbar_wait(&q_ready[t], 0u, abort_flag, p.status, 4);
-            // S_t(0)
-            if (ok) ok = mbar_wait(&k_full[0], 0u, abort_flag, p.status, 5);
-            if (ok) {
-                tc_fence_after();
-                for (int t = 0; t < 2; ++t)
-                    if (nkv[t] > 0) { issue_qk(t, 0); umma_commit(&s_full[t]); }
-                umma_commit(&k_empty[0]);
-            }
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const int st = j & 1, stn = (j + 1) & 1;
-                bool v_waited = false, k_waited = false;
-                for (int t = 0; t < 2 && ok; ++t) {
-                    if (j >= nkv[t]) continue;
-                    if (!mbar_wait(&p_full[t], j & 1, abort_flag, p.status, 6)) { ok = false; break; }
-                    if (!v_waited) {
-                        if (!mbar_wait(&v_full[st], (j >> 1) & 1, abort_flag, p.status, 7)) { ok = false; break; }
-                        v_waited = true;
-                    }
-                    tc_fence_after();
-                    issue_pv(t, st, j > 0 ? 1u : 0u);
-                    umma_commit(&o_done[t]);
-                    if (j + 1 < nkv[t]) {
-                        if (!k_waited) {
-                            if (!mbar_wait(&k_full[stn], ((j + 1) >> 1) & 1, abort_flag, p.status, 8)) { ok = false; break; }
-                            k_waited = true;
+            while (ok) {
+                const int slot = n_items & 1;
+                if (!mbar_wait(&item_full[slot], (n_items >> 1) & 1, abort_flag, p.status, 4)) break;
+                const int item = item_ring[slot];
+                mbar_arrive(&item_empty[slot]);
+                if (item < 0) break;
+                const Item g = item_geom(p, item);
+                const int nkv[2] = {g.nkv0, g.nkv1};
+                // S_t(0): tile 0 starts as soon as ITS Q tile is rewritten and ITS old O has been read out
+                {
+                    const uint32_t n0 = 2 * kv_use, st0 = n0 % kKVSlots;   // K of the item's first key tile
+                    bool k_waited = false;
+                    for (int t = 0; t < 2 && ok; ++t) {
+                        ok = mbar_wait(&q_ready[t], n_items & 1, abort_flag, p.status, 4);
+                        if (ok && n_items > 0) ok = mbar_wait(&o_free[t], (n_items - 1) & 1, abort_flag, p.status, 4);
+                        if (!ok) break;
+                        if (nkv[t] > 0) {
+                            if (!k_waited) {
+                                if (!mbar_wait(&kv_full[st0], (n0 / kKVSlots) & 1, abort_flag, p.status, 5)) { ok = false; break; }
+                                k_waited = true;
+                            }
                             tc_fence_after();
+                            issue_qk(t, st0);
+                            umma_commit(&s_full[t]);
                         }
-                        issue_qk(t, stn);
-                        umma_commit(&s_full[t]);
+                        if (nkv[t] <= 1) umma_commit(&q_empty[t]);   // that was tile t's only (or no) QK^T
                     }
+                    if (!ok) break;
+                    umma_commit(&kv_empty[st0]);
+                }
+                for (int j = 0; j < g.n_kv && ok; ++j) {
+                    const uint32_t nv = 2 * (kv_use + j) + 1, nk = nv + 1;   // load numbers of V_j and K_j+1
+                    const uint32_t st = nv % kKVSlots, stn = nk % kKVSlots;
+                    bool v_waited = false, k_waited = false;
+                    for (int t = 0; t < 2 && ok; ++t) {
+                        if (j >= nkv[t]) continue;
+                        if (!mbar_wait(&p_full[t], cp[t] & 1, abort_flag, p.status, 6)) { ok = false; break; }
+                        ++cp[t];
+                        if (!v_waited) {
+                            if (!mbar_wait(&kv_full[st], (nv / kKVSlots) & 1, abort_flag, p.status, 7)) { ok = false; break; }
+                            v_waited = true;
+                        }
+                        tc_fence_after();
+                        issue_pv(t, st, j > 0 ? 1u : 0u);
+                        umma_commit(&o_done[t]);
+                        if (j + 1 < nkv[t]) {
+                            if (!k_waited) {
+                                if (!mbar_wait(&kv_full[stn], (nk / kKVSlots) & 1, abort_flag, p.status, 8)) { ok = false; break; }
+                                k_waited = true;
+                                tc_fence_after();
+                            }
+                            issue_qk(t, stn);
+                            umma_commit(&s_full[t]);
+                            if (j + 2 == nkv[t]) umma_commit(&q_empty[t]);   // tile t's last QK^T: its Q tile is free
+                        }
+                    }
+                    if (!ok) break;
+                    umma_commit(&kv_empty[st]);                  // all PV of key tile j issued: V_j's slot is free
+                    if (k_waited) umma_commit(&kv_empty[stn]);   // all QK of key tile j+1 issued: K_j+1's slot is free
                 }
                 if (!ok) break;
-                umma_commit(&v_empty[st]);           // all PV of key tile j issued
-                if (k_waited) umma_commit(&k_empty[stn]);  // all QK of key tile j+1 issued
+                kv_use += static_cast<uint32_t>(g.n_kv);
+                ++n_items;
             }
         }
     } else {
@@ -286,50 +363,9 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const int t = (warp - 2) >> 2;             // 0: Q tile 0, 1: Q tile 1
         const int q = warp & 3;                    // TMEM lane quadrant
         const int r = q * 32 + lane;               // row within the tile
-        const int qt = qt0 + t;
-        const int my_nkv = (t == 0) ? n_kv_t0 : n_kv_t1;
-        const int row_g = qt * kT + r;             // query index within the sequence
         const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t tS = tmem_base + t * kT + lane_sel;
         const uint32_t tO = tmem_base + 2 * kT + t * kD + lane_sel;
-        bool ok = my_nkv > 0;
-        float rq = 0.f;
-        if (ok) ok = warp_wait(q_full, 0u, abort_flag, p.status, 9);
-        if (ok) {
-            // in-place rewrite of this thread's query row: qhat_d = fp16(q_d * rq_i * gq_d * gk_d)
-            // (|q * rq| <= sqrt(128), so fp16 is safe unless the gammas are huge: clamp to its range)
-            uint8_t* qrow = smem + kOffQ + t * kTileBytes + r * 128;
-            float ss = 0.f;
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
-                    ss += a * a + b * b;
-                }
-            }
-            rq = rsqrtf(ss * (1.f / kD) + p.eps);
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                uint4* ptr = reinterpret_cast<uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
-                const uint4 v = *ptr;
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                uint32_t o4[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float a = __uint_as_float(w[i] << 16) * rq * gprod[c * 8 + 2 * i];
-                    const float b = __uint_as_float(w[i] & 0xFFFF0000u) * rq * gprod[c * 8 + 2 * i + 1];
-                    o4[i] = pack_f16x2(fminf(fmaxf(a, -65504.f), 65504.f), fminf(fmaxf(b, -65504.f), 65504.f));
-                }
-                *ptr = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-            }
-            rq = p.scale_log2;   // the logits' only remaining factor: scale * log2(e), the same for every row
-            fence_proxy_async_smem();
-            mbar_arrive(&q_ready[t]);
-        }
-        const uint64_t rq2 = pack_f32x2(__float_as_uint(rq), __float_as_uint(rq));
         // Normalised queries and keys bound every logit: |qhat . khat| <= 128 * max_d |gq_d gk_d|
         // (Cauchy-Schwarz on rows of RMS <= 1).  When that bound is modest the softmax needs no running
         // maximum at all: exp2(x - bound) can neither overflow nor lose the row (p >= 2^(-2*bound)),
@@ -339,96 +375,149 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int d = 0; d < kD; ++d) gmax = fmaxf(gmax, fabsf(gprod[d]));
         const float bound = static_cast<float>(kD) * gmax * p.scale_log2;
         const bool fixed_ref = bound <= kFixedRefLimit;
-        float m_ref = fixed_ref ? bound : -INFINITY, l_sum = 0.f;
-        for (int j = 0; j < my_nkv && ok; ++j) {
-            if (!warp_wait(&s_full[t], j & 1, abort_flag, p.status, 10)) { ok = false; break; }
-            tc_fence_after();
-            uint32_t s[4][32];
+        const float rq = p.scale_log2;   // the logits' only remaining factor: scale * log2(e), the same for every row
+        const uint64_t rq2 = pack_f32x2(__float_as_uint(rq), __float_as_uint(rq));
+        uint32_t n_items = 0;
+        uint32_t cs = 0;   // s_full completions consumed by this group
+        uint32_t co = 0;   // PV (o_done) completions of earlier items of this group's tile
+        bool ok = true;
+        while (ok) {
+            const int slot = n_items & 1;
+            if (!warp_wait(&item_full[slot], (n_items >> 1) & 1, abort_flag, p.status, 9)) break;
+            const int item = item_ring[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&item_empty[slot]);
+            if (item < 0) break;
+            const Item g = item_geom(p, item);
+            const int my_nkv = (t == 0) ? g.nkv0 : g.nkv1;
+            const int qt = g.qt0 + t;
+            const int row_g = qt * kT + r;             // query index within the sequence
+            if (!warp_wait(&q_full[t], n_items & 1, abort_flag, p.status, 9)) break;
+            if (my_nkv > 0) {
+                // in-place rewrite of this thread's query row: qhat_d = fp16(q_d * rq_i * gq_d * gk_d)
+                // (|q * rq| <= sqrt(128), so fp16 is safe unless the gammas are huge: clamp to its range)
+                uint8_t* qrow = smem + kOffQ + t * kTileBytes + r * 128;
+                float ss = 0.f;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s[c]);
-            tmem_wait_ld();
-            const bool diag = p.causal && (j == qt);
-            if (diag || (j * kT + kT > p.S)) {  // diagonal tile or ragged last key tile only
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int col = c * 32 + i;
-                        if (!((!diag || col <= r) && (j * kT + col < p.S))) s[c][i] = 0xFF800000u;  // -inf
+                    for (int i = 0; i < 4; ++i) {
+                        const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
+                        ss += a * a + b * b;
                     }
                 }
-            }
-            // Running maximum with lazy repair -- skipped entirely when the logits are bounded a priori.
-            float o_scale = 1.f;
-            bool need = false;
-            if (!fixed_ref) {
-                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                const float rqi = rsqrtf(ss * (1.f / kD) + p.eps);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 16; ++c) {
+                    uint4* ptr = reinterpret_cast<uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
+                    const uint4 v = *ptr;
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                    uint32_t o4[4];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2)
-                        mx[(i >> 1) & 3] = max3(mx[(i >> 1) & 3], __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
+                    for (int i = 0; i < 4; ++i) {
+                        const float a = __uint_as_float(w[i] << 16) * rqi * gprod[c * 8 + 2 * i];
+                        const float b = __uint_as_float(w[i] & 0xFFFF0000u) * rqi * gprod[c * 8 + 2 * i + 1];
+                        o4[i] = pack_f16x2(fminf(fmaxf(a, -65504.f), 65504.f), fminf(fmaxf(b, -65504.f), 65504.f));
+                    }
+                    *ptr = make_uint4(o4[0], o4[1], o4[2], o4[3]);
                 }
-                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * rq;   // rq = scale * log2(e) > 0
-                need = m_tile > m_ref + kRescaleThreshold;
-                if (need) {
-                    o_scale = fast_exp2(m_ref - m_tile);  // 0 on the first tile (m_ref = -inf)
-                    l_sum *= o_scale;
-                    m_ref = m_tile;
-                }
+                fence_proxy_async_smem();
             }
-            // p = exp2(acc * scale*log2e - m_ref): packed FMA, two exp2, packed row sum (4 independent accumulators)
-            const uint64_t nm2 = pack_f32x2(__float_as_uint(-m_ref), __float_as_uint(-m_ref));
-            uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
-            uint32_t pk[64];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float a, b;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(s[c][2 * i], s[c][2 * i + 1]), rq2, nm2), a, b);
-                    const float p0 = fast_exp2(a), p1 = fast_exp2(b);
-                    acc2[i & 3] = add_f32x2(acc2[i & 3], pack_f32x2(__float_as_uint(p0), __float_as_uint(p1)));
-                    pk[c * 16 + i] = pack_bf16x2(p0, p1);
-                }
-            }
-            {
-                float a, b;
-                unpack_f32x2(add_f32x2(add_f32x2(acc2[0], acc2[1]), add_f32x2(acc2[2], acc2[3])), a, b);
-                l_sum += a + b;
-            }
-            // P (bf16) overwrites the first 64 columns of this thread's own S row
-            {
-                uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&pk[0]);
-                uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&pk[32]);
-                tmem_st32(tS, lo);
-                tmem_st32(tS + 32, hi);
-            }
-            // rescale the accumulated value when some row of this warp moved its reference maximum
-            if (j > 0 && __any_sync(0xffffffffu, need)) {
-                if (!warp_wait(&o_done[t], (j - 1) & 1, abort_flag, p.status, 12)) { ok = false; break; }
+            mbar_arrive(&q_ready[t]);   // every thread, every item (also when this tile has no work)
+            float m_ref = fixed_ref ? bound : -INFINITY, l_sum = 0.f;
+            for (int j = 0; j < my_nkv && ok; ++j) {
+                if (!warp_wait(&s_full[t], cs & 1, abort_flag, p.status, 10)) { ok = false; break; }
+                ++cs;
                 tc_fence_after();
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t ov[32];
-                    tmem_ld32(tO + c * 32, ov);
-                    tmem_wait_ld();
+                uint32_t s[4][32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * o_scale);
-                    tmem_st32(tO + c * 32, ov);
+                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s[c]);
+                tmem_wait_ld();
+                const bool diag = p.causal && (j == qt);
+                if (diag || (j * kT + kT > p.S)) {  // diagonal tile or ragged last key tile only
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int col = c * 32 + i;
+                            if (!((!diag || col <= r) && (j * kT + col < p.S))) s[c][i] = 0xFF800000u;  // -inf
+                        }
+                    }
                 }
+                // Running maximum with lazy repair -- skipped entirely when the logits are bounded a priori.
+                float o_scale = 1.f;
+                bool need = false;
+                if (!fixed_ref) {
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2)
+                            mx[(i >> 1) & 3] = max3(mx[(i >> 1) & 3], __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
+                    }
+                    const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * rq;   // rq = scale * log2(e) > 0
+                    need = m_tile > m_ref + kRescaleThreshold;
+                    if (need) {
+                        o_scale = fast_exp2(m_ref - m_tile);  // 0 on the first tile (m_ref = -inf)
+                        l_sum *= o_scale;
+                        m_ref = m_tile;
+                    }
+                }
+                // p = exp2(acc * scale*log2e - m_ref): packed FMA, two exp2, packed row sum (4 independent accumulators)
+                const uint64_t nm2 = pack_f32x2(__float_as_uint(-m_ref), __float_as_uint(-m_ref));
+                uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
+                uint32_t pk[64];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float a, b;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(s[c][2 * i], s[c][2 * i + 1]), rq2, nm2), a, b);
+                        const float p0 = fast_exp2(a), p1 = fast_exp2(b);
+                        acc2[i & 3] = add_f32x2(acc2[i & 3], pack_f32x2(__float_as_uint(p0), __float_as_uint(p1)));
+                        pk[c * 16 + i] = pack_bf16x2(p0, p1);
+                    }
+                }
+                {
+                    float a, b;
+                    unpack_f32x2(add_f32x2(add_f32x2(acc2[0], acc2[1]), add_f32x2(acc2[2], acc2[3])), a, b);
+                    l_sum += a + b;
+                }
+                // P (bf16) overwrites the first 64 columns of this thread's own S row
+                {
+                    uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&pk[0]);
+                    uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&pk[32]);
+                    tmem_st32(tS, lo);
+                    tmem_st32(tS + 32, hi);
+                }
+                // rescale the accumulated value when some row of this warp moved its reference maximum
+                if (j > 0 && __any_sync(0xffffffffu, need)) {
+                    if (!warp_wait(&o_done[t], (co + j - 1) & 1, abort_flag, p.status, 12)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t ov[32];
+                        tmem_ld32(tO + c * 32, ov);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * o_scale);
+                        tmem_st32(tO + c * 32, ov);
+                    }
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full[t]);
             }
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&p_full[t]);
-        }
-        if (ok && my_nkv > 0) {
-            // epilogue: O / l
-            if (warp_wait(&o_done[t], (my_nkv - 1) & 1, abort_flag, p.status, 13)) {
+            if (!ok) break;
+            // epilogue: read O out of TMEM (then the next item may overwrite it), scale by 1/l, store
+            if (my_nkv > 0) {
+                if (!warp_wait(&o_done[t], (co + my_nkv - 1) & 1, abort_flag, p.status, 13)) break;
                 tc_fence_after();
                 const float inv = 1.f / l_sum;
-                __nv_bfloat16* orow = p.O + (static_cast<size_t>(bh) * p.S + row_g) * kD;
+                uint4* orow = reinterpret_cast<uint4*>(p.O + (static_cast<size_t>(g.bh) * p.S + row_g) * kD);
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
                     uint32_t ov[32];
@@ -442,11 +531,16 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                             o.y = pack_bf16x2(__uint_as_float(ov[v * 8 + 2]) * inv, __uint_as_float(ov[v * 8 + 3]) * inv);
                             o.z = pack_bf16x2(__uint_as_float(ov[v * 8 + 4]) * inv, __uint_as_float(ov[v * 8 + 5]) * inv);
                             o.w = pack_bf16x2(__uint_as_float(ov[v * 8 + 6]) * inv, __uint_as_float(ov[v * 8 + 7]) * inv);
-                            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = o;
+                            orow[c * 4 + v] = o;
                         }
                     }
                 }
+                co += static_cast<uint32_t>(my_nkv);
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_free[t]);   // every item, also when this tile had no work
+            ++n_items;
         }
     }
     tc_fence_before();
@@ -520,7 +614,9 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     p.eps = eps;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = reinterpret_cast<uint32_t*>(w);
-    const unsigned grid = static_cast<unsigned>(BH * n_pairs);
+    p.header = reinterpret_cast<uint32_t*>(w);
+    p.total_items = static_cast<int>(BH * n_pairs);
+    const unsigned grid = static_cast<unsigned>(p.total_items < di.num_sms ? p.total_items : di.num_sms);
     EF_CUDA_CHECK(launch_pdl(attn::qknorm_attn_kernel, dim3(grid), dim3(attn::kThreads), attn::kSmemBytes, s, tmQ, tmK, tmV, p));
     return EF_OK;
 }

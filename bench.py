@@ -110,20 +110,19 @@ def run_ours(args):
 
     import paper_2609_12330_b200 as ef
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2609_12330_b200 import replicas
+
+    info = replicas.rank_info()
+    rank, world, local = info.rank, info.world, info.local
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    replicas.init_process_group(info, "nccl", device=torch.device("cuda", local))
     ef.lib()  # fail loudly if the extension is missing
 
     host, dev, params, wss, outs = {}, {}, {}, {}, {}
     for prog in wl.PROGRAMS:
-        p, t = wl.make_inputs(prog, seed=rank, size="full")
+        p, t = wl.make_inputs(prog, seed=replicas.replica_seed(info), size="full")
         params[prog] = p
         host[prog] = {k: wl.bf16_bits_to_torch(v).pin_memory() for k, v in t.items()}
         dev[prog] = {k: v.to("cuda", non_blocking=True) for k, v in host[prog].items()}
@@ -141,17 +140,10 @@ def run_ours(args):
             ef.run(prog, params[prog], dev[prog], wss[prog], out=outs[prog])
 
     def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(info, torch.cuda.synchronize)
 
     def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        tns = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tns, op=dist.ReduceOp.MAX)
-        return float(tns.item())
+        return replicas.max_over_ranks(info, ms, device="cuda")
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -174,7 +166,7 @@ def run_ours(args):
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     clocks = sampler.stop(t0, t1)
     ms_per_step = ms_total / args.steps
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = replicas.aggregate_rate(info, step_flops, ms_per_step) / 1e12
 
     # ---- per-program latency: median over CUDA-graph replays of back-to-back calls (the paper's
     #      protocol, Section 7.1), rotating over enough input copies that > 256 MB are touched between
@@ -253,7 +245,7 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / n_e2e
-    e2e = {"value": round(world * step_flops / (e2e_ms * 1e-3) / 1e12, 3), "unit": "TFLOP/s", "ms_per_step": round(e2e_ms, 3),
+    e2e = {"value": round(replicas.aggregate_rate(info, step_flops, e2e_ms) / 1e12, 3), "unit": "TFLOP/s", "ms_per_step": round(e2e_ms, 3),
            "steps": n_e2e, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes}
     for prog in wl.PROGRAMS:
         wss[prog].check()
@@ -275,8 +267,7 @@ def run_ours(args):
         line["cpu_baseline"] = cpu_baseline()
     if rank == 0:
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.destroy_process_group(info)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -315,7 +306,9 @@ def cpu_baseline():
 
 
 def run_reference(args):
-    if int(os.environ.get("RANK", "0")) != 0:
+    from paper_2609_12330_b200 import replicas
+
+    if not replicas.rank_info().is_root:   # rank 0 alone runs and prints the oracle arm
         return
     import oracle
 

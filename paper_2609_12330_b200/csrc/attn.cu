@@ -40,7 +40,7 @@ constexpr int kD = 128;
 constexpr int kT = 128;                           // tile edge (queries and keys)
 constexpr int kHalfBytes = kT * 128;              // [128 rows][64 d] bf16, 128B swizzle
 constexpr int kTileBytes = 2 * kHalfBytes;        // 32 KiB
-constexpr int kKVSlots = 5;                        // one ring for K and V tiles: K_j, V_j, K_j+1, V_j+1, K_j+2
+constexpr int kKVSlots = 4;                        // one ring for K and V tiles: K_j, V_j, K_j+1, V_j+1, K_j+2
 constexpr int kThreads = 320;
 constexpr int kSoftmaxThreads = 128;
 constexpr uint32_t kTmemCols = 512;               // S0 | S1 | O0 | O1, 128 fp32 columns each
@@ -62,6 +62,7 @@ struct Params {
     int BH, S, nq, n_pairs, causal;
     float eps, scale_log2;
     int total_items;
+    int o_vec8;           // O is 32-byte aligned: the epilogue may use 256-bit stores
     uint32_t* status;
     uint32_t* header;   // workspace header: work counter / done counter for the persistent grid
 };
@@ -99,6 +100,11 @@ __device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
     uint64_t d;
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
+}
+__device__ __forceinline__ void st_global_v8(void* dst, const uint32_t* v) {   // 32-byte aligned destination
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+                 "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -148,18 +154,22 @@ __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16*
 struct Item {
     int bh, qt0, n_kv, nkv0, nkv1;
 };
-__device__ __forceinline__ Item item_geom(const Params& p, int item) {
+// geometry of the pair whose first Q tile is qt0 (no division: the consumers' per-item path)
+__device__ __forceinline__ Item item_from(const Params& p, int bh, int qt0) {
     Item g;
-    const int pair = p.n_pairs - 1 - item / p.BH;
-    g.bh = item - (item / p.BH) * p.BH;
-    g.qt0 = 2 * pair;
-    const int qt1 = g.qt0 + 1;
+    g.bh = bh;
+    g.qt0 = qt0;
+    const int qt1 = qt0 + 1;
     const bool has_q1 = qt1 < p.nq;
-    const int q_last = has_q1 ? qt1 : g.qt0;
+    const int q_last = has_q1 ? qt1 : qt0;
     g.n_kv = p.causal ? (q_last + 1) : p.nq;                       // key tiles the pair visits
-    g.nkv0 = p.causal ? (g.qt0 + 1) : p.nq;                        // ... and each of its two Q tiles
+    g.nkv0 = p.causal ? (qt0 + 1) : p.nq;                          // ... and each of its two Q tiles
     g.nkv1 = has_q1 ? (p.causal ? (qt1 + 1) : p.nq) : 0;
     return g;
+}
+__device__ __forceinline__ Item item_geom(const Params& p, int item) {
+    const int pair = p.n_pairs - 1 - item / p.BH;
+    return item_from(p, item - (item / p.BH) * p.BH, 2 * pair);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -180,8 +190,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     uint64_t* o_free = bars + 22;            // [2]  softmax group t -> MMA (O_t read out: may be overwritten)
     uint64_t* item_full = bars + 24;         // [2]  TMA -> everyone (work item published)
     uint64_t* item_empty = bars + 26;        // [2]  everyone -> TMA (item slot read)
-    int* item_ring = reinterpret_cast<int*>(bars + 28);   // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 29);
+    int2* item_ring = reinterpret_cast<int2*>(bars + 28);   // [2]  {batch*head, first Q tile}; x < 0: no more work
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 30);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -221,11 +231,11 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 const int slot = n_items & 1;
                 if (!mbar_wait(&item_empty[slot], ((n_items >> 1) & 1) ^ 1u, abort_flag, p.status, 1)) break;
                 const bool valid = item < static_cast<uint32_t>(p.total_items);
-                item_ring[slot] = valid ? static_cast<int>(item) : -1;
+                const Item g = item_geom(p, valid ? static_cast<int>(item) : 0);
+                item_ring[slot] = valid ? make_int2(g.bh, g.qt0) : make_int2(-1, 0);
                 mbar_arrive(&item_full[slot]);
                 if (!valid) break;
                 const uint32_t next = atomicAdd(&p.header[kWorkCounterWord], 1u);   // latency hides behind the copies
-                const Item g = item_geom(p, static_cast<int>(item));
                 // Q tile t of the new item goes in as soon as the previous item's last QK^T of tile t is done
                 // (tile 0 finishes one key tile earlier than tile 1 under the causal mask), so the load is
                 // hidden behind the previous item's tail.  Order: Q0, K(0), Q1, V(0), then the remaining K/V.
@@ -296,10 +306,10 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             while (ok) {
                 const int slot = n_items & 1;
                 if (!mbar_wait(&item_full[slot], (n_items >> 1) & 1, abort_flag, p.status, 4)) break;
-                const int item = item_ring[slot];
+                const int2 item = item_ring[slot];
                 mbar_arrive(&item_empty[slot]);
-                if (item < 0) break;
-                const Item g = item_geom(p, item);
+                if (item.x < 0) break;
+                const Item g = item_from(p, item.x, item.y);
                 const int nkv[2] = {g.nkv0, g.nkv1};
                 // S_t(0): tile 0 starts as soon as ITS Q tile is rewritten and ITS old O has been read out
                 {
@@ -384,11 +394,11 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         while (ok) {
             const int slot = n_items & 1;
             if (!warp_wait(&item_full[slot], (n_items >> 1) & 1, abort_flag, p.status, 9)) break;
-            const int item = item_ring[slot];
+            const int2 item = item_ring[slot];
             __syncwarp();
             if (lane == 0) mbar_arrive(&item_empty[slot]);
-            if (item < 0) break;
-            const Item g = item_geom(p, item);
+            if (item.x < 0) break;
+            const Item g = item_from(p, item.x, item.y);
             const int my_nkv = (t == 0) ? g.nkv0 : g.nkv1;
             const int qt = g.qt0 + t;
             const int row_g = qt * kT + r;             // query index within the sequence
@@ -397,11 +407,12 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 // in-place rewrite of this thread's query row: qhat_d = fp16(q_d * rq_i * gq_d * gk_d)
                 // (|q * rq| <= sqrt(128), so fp16 is safe unless the gammas are huge: clamp to its range)
                 uint8_t* qrow = smem + kOffQ + t * kTileBytes + r * 128;
+                uint4 v[16];   // the whole row stays in registers between the two passes
                 float ss = 0.f;
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
-                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                    v[c] = *reinterpret_cast<const uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
+                    const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
@@ -409,20 +420,29 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     }
                 }
                 const float rqi = rsqrtf(ss * (1.f / kD) + p.eps);
+                const float4* g4 = reinterpret_cast<const float4*>(gprod);
+                auto rewrite = [&](const bool clamp) {
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    uint4* ptr = reinterpret_cast<uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
-                    const uint4 v = *ptr;
-                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                    uint32_t o4[4];
+                    for (int c = 0; c < 16; ++c) {
+                        const float4 ga = g4[2 * c], gb = g4[2 * c + 1];
+                        const float gg[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+                        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                        uint32_t o4[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float a = __uint_as_float(w[i] << 16) * rqi * gprod[c * 8 + 2 * i];
-                        const float b = __uint_as_float(w[i] & 0xFFFF0000u) * rqi * gprod[c * 8 + 2 * i + 1];
-                        o4[i] = pack_f16x2(fminf(fmaxf(a, -65504.f), 65504.f), fminf(fmaxf(b, -65504.f), 65504.f));
+                        for (int i = 0; i < 4; ++i) {
+                            float a = __uint_as_float(w[i] << 16) * rqi * gg[2 * i];
+                            float b = __uint_as_float(w[i] & 0xFFFF0000u) * rqi * gg[2 * i + 1];
+                            if (clamp) {
+                                a = fminf(fmaxf(a, -65504.f), 65504.f);
+                                b = fminf(fmaxf(b, -65504.f), 65504.f);
+                            }
+                            o4[i] = pack_f16x2(a, b);
+                        }
+                        *reinterpret_cast<uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4)) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
                     }
-                    *ptr = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-                }
+                };
+                // |q * rq| <= sqrt(128) per element, so only huge gammas can leave the fp16 range
+                if (gmax * 11.32f > 65504.f) rewrite(true); else rewrite(false);
                 fence_proxy_async_smem();
             }
             mbar_arrive(&q_ready[t]);   // every thread, every item (also when this tile has no work)
@@ -517,21 +537,31 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 if (!warp_wait(&o_done[t], (co + my_nkv - 1) & 1, abort_flag, p.status, 13)) break;
                 tc_fence_after();
                 const float inv = 1.f / l_sum;
-                uint4* orow = reinterpret_cast<uint4*>(p.O + (static_cast<size_t>(g.bh) * p.S + row_g) * kD);
+                uint8_t* orow = reinterpret_cast<uint8_t*>(p.O + (static_cast<size_t>(g.bh) * p.S + row_g) * kD);
+                // two rounds of 64 columns: both TMEM loads of a round in flight, then 32-byte stores (a lane
+                // fills whole sectors; a 16-byte store pattern leaves every sector half written per instruction)
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t ov[32];
-                    tmem_ld32(tO + c * 32, ov);
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t ov[2][32];
+                    tmem_ld32(tO + half * 64, ov[0]);
+                    tmem_ld32(tO + half * 64 + 32, ov[1]);
                     tmem_wait_ld();
                     if (row_g < p.S) {
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(ov[v * 8 + 0]) * inv, __uint_as_float(ov[v * 8 + 1]) * inv);
-                            o.y = pack_bf16x2(__uint_as_float(ov[v * 8 + 2]) * inv, __uint_as_float(ov[v * 8 + 3]) * inv);
-                            o.z = pack_bf16x2(__uint_as_float(ov[v * 8 + 4]) * inv, __uint_as_float(ov[v * 8 + 5]) * inv);
-                            o.w = pack_bf16x2(__uint_as_float(ov[v * 8 + 6]) * inv, __uint_as_float(ov[v * 8 + 7]) * inv);
-                            orow[c * 4 + v] = o;
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                pk[i] = pack_bf16x2(__uint_as_float(ov[c][2 * i]) * inv, __uint_as_float(ov[c][2 * i + 1]) * inv);
+                            uint8_t* dst = orow + half * 128 + c * 64;
+                            if (p.o_vec8) {
+                                st_global_v8(dst, &pk[0]);
+                                st_global_v8(dst + 32, &pk[8]);
+                            } else {
+#pragma unroll
+                                for (int v = 0; v < 4; ++v)
+                                    reinterpret_cast<uint4*>(dst)[v] = make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
+                            }
                         }
                     }
                 }
@@ -616,6 +646,7 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     p.status = reinterpret_cast<uint32_t*>(w);
     p.header = reinterpret_cast<uint32_t*>(w);
     p.total_items = static_cast<int>(BH * n_pairs);
+    p.o_vec8 = aligned(O, 32) ? 1 : 0;
     const unsigned grid = static_cast<unsigned>(p.total_items < di.num_sms ? p.total_items : di.num_sms);
     EF_CUDA_CHECK(launch_pdl(attn::qknorm_attn_kernel, dim3(grid), dim3(attn::kThreads), attn::kSmemBytes, s, tmQ, tmK, tmV, p));
     return EF_OK;

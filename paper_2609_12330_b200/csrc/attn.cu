@@ -42,7 +42,6 @@ constexpr int kHalfBytes = kT * 128;              // [128 rows][64 d] bf16, 128B
 constexpr int kTileBytes = 2 * kHalfBytes;        // 32 KiB
 constexpr int kKVSlots = 4;                        // one ring for K and V tiles: K_j, V_j, K_j+1, V_j+1, K_j+2
 constexpr int kThreads = 320;
-constexpr int kSoftmaxThreads = 128;
 constexpr uint32_t kTmemCols = 512;               // S0 | S1 | O0 | O1, 128 fp32 columns each
 // shared memory map (offsets from the 1024-aligned base)
 constexpr int kOffQ = 0;                                          // 2 tiles
@@ -113,10 +112,14 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// pre-pass: Khat[row] = fp16(K[row] * rsqrt(mean_d K[row][d]^2 + eps)); 16 threads per key row,
-// one 16-byte piece each, so every load of the grid is in flight at once
+// pre-pass: Khat[row][d] = fp16(K[row][d] * rsqrt(mean_d K[row][d]^2 + eps) * gq[d] * gk[d]): both gammas ride
+// on the keys (the logit only needs their product), so the query side needs no per-column factor.  16 threads
+// per key row, one 16-byte piece each, so every load of the grid is in flight at once.  |k * rk| <= sqrt(128);
+// the clamp only matters for huge gammas.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16* __restrict__ K,
+                                                            const __nv_bfloat16* __restrict__ gamma_q,
+                                                            const __nv_bfloat16* __restrict__ gamma_k,
                                                             __nv_bfloat16* __restrict__ Khat, long long rows, float eps) {
     pdl_launch_dependents();
     pdl_wait();
@@ -126,6 +129,9 @@ __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16*
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (live) v = __ldg(reinterpret_cast<const uint4*>(K + row * kD) + sub);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float g[8];   // gq*gk of this thread's 8 columns (2-byte loads: the gammas need no 16-byte alignment)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) g[i] = __bfloat162float(gamma_q[sub * 8 + i]) * __bfloat162float(gamma_k[sub * 8 + i]);
     float lo[4], hi[4], ss = 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -137,12 +143,12 @@ __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16*
     for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     const float rk = rsqrtf(ss * (1.f / kD) + eps);
     if (live) {
-        uint4 o4;
-        o4.x = pack_f16x2(lo[0] * rk, hi[0] * rk);
-        o4.y = pack_f16x2(lo[1] * rk, hi[1] * rk);
-        o4.z = pack_f16x2(lo[2] * rk, hi[2] * rk);
-        o4.w = pack_f16x2(lo[3] * rk, hi[3] * rk);
-        reinterpret_cast<uint4*>(Khat + row * kD)[sub] = o4;
+        uint32_t o4[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            o4[i] = pack_f16x2(fminf(fmaxf(lo[i] * rk * g[2 * i], -65504.f), 65504.f), fminf(fmaxf(hi[i] * rk * g[2 * i + 1], -65504.f), 65504.f));
+        }
+        reinterpret_cast<uint4*>(Khat + row * kD)[sub] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
     }
 }
 
@@ -199,7 +205,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     if (threadIdx.x == 0) {
         for (int t = 0; t < 2; ++t) {
             mbar_init(&q_full[t], 1); mbar_init(&q_empty[t], 1);
-            mbar_init(&q_ready[t], kSoftmaxThreads);
+            mbar_init(&q_ready[t], 4);
             mbar_init(&s_full[t], 1); mbar_init(&p_full[t], 4); mbar_init(&o_done[t], 1); mbar_init(&o_free[t], 4);
             mbar_init(&item_full[t], 1); mbar_init(&item_empty[t], 9);   // MMA thread + 8 softmax warps
         }
@@ -404,11 +410,11 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const int row_g = qt * kT + r;             // query index within the sequence
             if (!warp_wait(&q_full[t], n_items & 1, abort_flag, p.status, 9)) break;
             if (my_nkv > 0) {
-                // in-place rewrite of this thread's query row: qhat_d = fp16(q_d * rq_i * gq_d * gk_d)
-                // (|q * rq| <= sqrt(128), so fp16 is safe unless the gammas are huge: clamp to its range)
+                // in-place rewrite of this thread's query row: qhat_d = fp16(q_d * rq_i); |q * rq| <= sqrt(128)
+                // whatever the scale of q, so fp16 is safe (the gammas ride on the keys)
                 uint8_t* qrow = smem + kOffQ + t * kTileBytes + r * 128;
                 uint4 v[16];   // the whole row stays in registers between the two passes
-                float ss = 0.f;
+                float ss4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     v[c] = *reinterpret_cast<const uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4));
@@ -416,36 +422,23 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
-                        ss += a * a + b * b;
+                        ss4[i] = fmaf(a, a, fmaf(b, b, ss4[i]));
                     }
                 }
-                const float rqi = rsqrtf(ss * (1.f / kD) + p.eps);
-                const float4* g4 = reinterpret_cast<const float4*>(gprod);
-                auto rewrite = [&](const bool clamp) {
+                const float rqi = rsqrtf(((ss4[0] + ss4[1]) + (ss4[2] + ss4[3])) * (1.f / kD) + p.eps);
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float4 ga = g4[2 * c], gb = g4[2 * c + 1];
-                        const float gg[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
-                        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-                        uint32_t o4[4];
+                for (int c = 0; c < 16; ++c) {
+                    const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                    uint32_t o4[4];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            float a = __uint_as_float(w[i] << 16) * rqi * gg[2 * i];
-                            float b = __uint_as_float(w[i] & 0xFFFF0000u) * rqi * gg[2 * i + 1];
-                            if (clamp) {
-                                a = fminf(fmaxf(a, -65504.f), 65504.f);
-                                b = fminf(fmaxf(b, -65504.f), 65504.f);
-                            }
-                            o4[i] = pack_f16x2(a, b);
-                        }
-                        *reinterpret_cast<uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4)) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-                    }
-                };
-                // |q * rq| <= sqrt(128) per element, so only huge gammas can leave the fp16 range
-                if (gmax * 11.32f > 65504.f) rewrite(true); else rewrite(false);
+                    for (int i = 0; i < 4; ++i)
+                        o4[i] = pack_f16x2(__uint_as_float(w[i] << 16) * rqi, __uint_as_float(w[i] & 0xFFFF0000u) * rqi);
+                    *reinterpret_cast<uint4*>(qrow + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4)) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+                }
                 fence_proxy_async_smem();
             }
-            mbar_arrive(&q_ready[t]);   // every thread, every item (also when this tile has no work)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&q_ready[t]);   // every warp, every item (also when this tile has no work)
             float m_ref = fixed_ref ? bound : -INFINITY, l_sum = 0.f;
             for (int j = 0; j < my_nkv && ok; ++j) {
                 if (!warp_wait(&s_full[t], cs & 1, abort_flag, p.status, 10)) { ok = false; break; }
@@ -634,7 +627,8 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
         const long long blocks = (rows * 16 + 255) / 256;
         if (blocks > 0x7fffffffLL) return EF_ERR_UNSUPPORTED;
         EF_CUDA_CHECK(launch_pdl(attn::key_normalize_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s,
-                                 static_cast<const __nv_bfloat16*>(K), Khat, rows, eps));
+                                 static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(gamma_q),
+                                 static_cast<const __nv_bfloat16*>(gamma_k), Khat, rows, eps));
     }
     attn::Params p;
     p.gamma_q = static_cast<const __nv_bfloat16*>(gamma_q);

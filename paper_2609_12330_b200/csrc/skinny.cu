@@ -400,6 +400,15 @@ ef_status launch(const void* X, const void* gamma, const void* W0, const void* W
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
     int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
     if (grid > kMaxGrid) grid = kMaxGrid;
+    if (pl.total_units / grid < 8) {
+        // Few units per block: the call is latency-bound, and ranges that straddle n-tile boundaries add partial
+        // slots and arrivals.  Cut every n tile into the same number s of k ranges instead (s divides k_blocks)
+        // as long as that keeps at least half of the blocks.
+        int s = 0;
+        for (int d = 1; d <= pl.k_blocks; ++d)
+            if (pl.k_blocks % d == 0 && static_cast<long long>(pl.n_tiles) * d <= grid) s = d;
+        if (s > 0 && pl.n_tiles * s * 2 >= grid) grid = pl.n_tiles * s;
+    }
     p.base = pl.total_units / grid;
     p.rem = pl.total_units % grid;
     p.stages = pl.stages;

@@ -42,6 +42,7 @@ constexpr int kHalfBytes = kT * 128;              // [128 rows][64 d] bf16, 128B
 constexpr int kTileBytes = 2 * kHalfBytes;        // 32 KiB
 constexpr int kKVSlots = 4;                        // one ring for K and V tiles: K_j, V_j, K_j+1, V_j+1, K_j+2
 constexpr int kThreads = 320;
+constexpr int kKeyRowsPerThread = 4;               // pre-pass: key rows per thread
 constexpr uint32_t kTmemCols = 512;               // S0 | S1 | O0 | O1, 128 fp32 columns each
 // shared memory map (offsets from the 1024-aligned base)
 constexpr int kOffQ = 0;                                          // 2 tiles
@@ -124,31 +125,39 @@ __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16*
     pdl_launch_dependents();
     pdl_wait();
     const int sub = threadIdx.x & 15;
-    const long long row = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 4;
-    const bool live = row < rows;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (live) v = __ldg(reinterpret_cast<const uint4*>(K + row * kD) + sub);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     float g[8];   // gq*gk of this thread's 8 columns (2-byte loads: the gammas need no 16-byte alignment)
 #pragma unroll
     for (int i = 0; i < 8; ++i) g[i] = __bfloat162float(gamma_q[sub * 8 + i]) * __bfloat162float(gamma_k[sub * 8 + i]);
-    float lo[4], hi[4], ss = 0.f;
+    // kKeyRowsPerThread rows per thread, 16 rows apart: all of a thread's loads are issued before the first use
+    const long long row0 = static_cast<long long>(blockIdx.x) * (16 * kKeyRowsPerThread) + (threadIdx.x >> 4);
+    uint4 v[kKeyRowsPerThread];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        lo[i] = __uint_as_float(w[i] << 16);
-        hi[i] = __uint_as_float(w[i] & 0xFFFF0000u);
-        ss += lo[i] * lo[i] + hi[i] * hi[i];
+    for (int u = 0; u < kKeyRowsPerThread; ++u) {
+        const long long row = row0 + 16 * u;
+        v[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (row < rows) v[u] = __ldg(reinterpret_cast<const uint4*>(K + row * kD) + sub);
     }
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    const float rk = rsqrtf(ss * (1.f / kD) + eps);
-    if (live) {
-        uint32_t o4[4];
+    for (int u = 0; u < kKeyRowsPerThread; ++u) {
+        const long long row = row0 + 16 * u;
+        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+        float lo[4], hi[4], ss = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            o4[i] = pack_f16x2(fminf(fmaxf(lo[i] * rk * g[2 * i], -65504.f), 65504.f), fminf(fmaxf(hi[i] * rk * g[2 * i + 1], -65504.f), 65504.f));
+            lo[i] = __uint_as_float(w[i] << 16);
+            hi[i] = __uint_as_float(w[i] & 0xFFFF0000u);
+            ss += lo[i] * lo[i] + hi[i] * hi[i];
         }
-        reinterpret_cast<uint4*>(Khat + row * kD)[sub] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        const float rk = rsqrtf(ss * (1.f / kD) + eps);
+        if (row < rows) {
+            uint32_t o4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                o4[i] = pack_f16x2(fminf(fmaxf(lo[i] * rk * g[2 * i], -65504.f), 65504.f), fminf(fmaxf(hi[i] * rk * g[2 * i + 1], -65504.f), 65504.f));
+            reinterpret_cast<uint4*>(Khat + row * kD)[sub] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+        }
     }
 }
 
@@ -624,7 +633,7 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     {
         const long long rows = BH * S;
-        const long long blocks = (rows * 16 + 255) / 256;
+        const long long blocks = (rows + 16 * attn::kKeyRowsPerThread - 1) / (16 * attn::kKeyRowsPerThread);
         if (blocks > 0x7fffffffLL) return EF_ERR_UNSUPPORTED;
         EF_CUDA_CHECK(launch_pdl(attn::key_normalize_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s,
                                  static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(gamma_q),

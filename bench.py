@@ -32,9 +32,9 @@ import workloads as wl  # noqa: E402
 METRIC = "us/call and TFLOP/s (GB/s for decode) per fused program, % of B200 roofline"
 UNIT = "TFLOP/s (algorithmic flops of one step = all five programs / step time; per-program us/call, TFLOP/s, GB/s in 'programs')"
 BOUND = {"rmsnorm_matmul": "hbm", "gated_mlp": "hbm", "gqa_decode": "hbm", "qknorm_attn": "tensor", "lora_linear": "tensor",
-         "rmsnorm_gated_mlp": "hbm"}
+         "rmsnorm_gated_mlp": "hbm", "gqa_decode_varlen": "hbm"}
 KERNELS_PER_CALL = {"rmsnorm_matmul": 1, "gated_mlp": 1, "gqa_decode": 1, "qknorm_attn": 2, "lora_linear": 2,
-                    "rmsnorm_gated_mlp": 1}
+                    "rmsnorm_gated_mlp": 1, "gqa_decode_varlen": 1}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -175,25 +175,30 @@ def run_ours(args):
     programs = {}
     gstream = torch.cuda.Stream()
     calls_per_graph = 20
-    for prog in wl.EXTRA_PROGRAMS:   # programs beyond the five configs of a step: measured the same way, outside the step
-        pp, tt = wl.make_inputs(prog, seed=rank, size="full")
-        params[prog] = pp
-        host[prog] = {k: wl.bf16_bits_to_torch(v) for k, v in tt.items()}
-        dev[prog] = {k: v.to("cuda") for k, v in host[prog].items()}
-        wss[prog] = ef.Workspace(ef.workspace_bytes(prog, pp))
-        outs[prog] = ef.run(prog, pp, dev[prog], wss[prog])
-        work[prog] = wl.algorithmic_work(prog, pp)
-    for prog in wl.PROGRAMS + wl.EXTRA_PROGRAMS:
-        nbytes = sum(v.numel() * 2 for v in host[prog].values())
+    # programs and shapes beyond the five configs of a step: measured the same way, outside the step
+    extras = [(q, q, {}) for q in wl.EXTRA_PROGRAMS] + [("gqa_decode[B=1]", "gqa_decode", {"B": 1}),
+                                                        ("gqa_decode[B=16]", "gqa_decode", {"B": 16})]
+    impl = {q: q for q in wl.PROGRAMS}   # key in `programs` -> entry point
+    for key, prog, over in extras:
+        pp, tt = wl.make_inputs(prog, seed=rank, size="full", **over)
+        impl[key] = prog
+        params[key] = pp
+        host[key] = {k: wl.to_torch(k, v) for k, v in tt.items()}
+        dev[key] = {k: v.to("cuda") for k, v in host[key].items()}
+        wss[key] = ef.Workspace(ef.workspace_bytes(prog, pp))
+        outs[key] = ef.run(prog, pp, dev[key], wss[key])
+        work[key] = wl.algorithmic_work(prog, pp)
+    for prog in list(wl.PROGRAMS) + [e[0] for e in extras]:
+        nbytes = sum(v.numel() * v.element_size() for v in host[prog].values())
         nsets = int(min(40, max(2, 256e6 // nbytes + 1)))
         sets = [dev[prog]] + [{k: v.clone() for k, v in dev[prog].items()} for _ in range(nsets - 1)]
         with torch.cuda.stream(gstream):
             for i in range(3):
-                ef.run(prog, params[prog], sets[i % nsets], wss[prog], out=outs[prog])
+                ef.run(impl[prog], params[prog], sets[i % nsets], wss[prog], out=outs[prog])
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=gstream):
                 for i in range(calls_per_graph):
-                    ef.run(prog, params[prog], sets[i % nsets], wss[prog], out=outs[prog])
+                    ef.run(impl[prog], params[prog], sets[i % nsets], wss[prog], out=outs[prog])
             for _ in range(3):
                 graph.replay()
             gstream.synchronize()
@@ -208,7 +213,7 @@ def run_ours(args):
             for i in range(10):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(gstream)
-                ef.run(prog, params[prog], sets[i % nsets], wss[prog], out=outs[prog])
+                ef.run(impl[prog], params[prog], sets[i % nsets], wss[prog], out=outs[prog])
                 b.record(gstream); gstream.synchronize()
                 ss.append(a.elapsed_time(b) * 1e3)
             warm_us = None
@@ -216,7 +221,7 @@ def run_ours(args):
                 wgraph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(wgraph, stream=gstream):
                     for i in range(calls_per_graph):
-                        ef.run(prog, params[prog], sets[0], wss[prog], out=outs[prog])
+                        ef.run(impl[prog], params[prog], sets[0], wss[prog], out=outs[prog])
                 for _ in range(3):
                     wgraph.replay()
                 gstream.synchronize()
@@ -232,20 +237,20 @@ def run_ours(args):
         w = work[prog]
         tf, gb = w["flops"] / us / 1e6, w["bytes"] / us / 1e3
         entry = {"us_per_call": round(us, 2), "us_min": round(float(np.min(ts)), 2), "tflops": round(tf, 1), "gbs": round(gb, 1),
-                 "bound": BOUND[prog], "kernels": KERNELS_PER_CALL[prog], "input_copies": nsets,
+                 "bound": BOUND[impl[prog]], "kernels": KERNELS_PER_CALL[impl[prog]], "input_copies": nsets,
                  "us_single_launch": round(float(np.median(ss)), 2),
                  "frac_hbm_measured": round(gb / peaks["hbm_gbs"], 4), "frac_tensor_sustained": round(tf / peaks["bf16_tflops_sustained"], 4),
                  "frac_hbm_nominal": round(gb / 8000.0, 4), "frac_tensor_nominal": round(tf / 2250.0, 4)}
         if warm_us is not None:
             entry["us_per_call_warm_l2"] = round(warm_us, 2)
-        if BOUND[prog] == "hbm":
+        if BOUND[impl[prog]] == "hbm":
             entry["frac"] = round(gb / peaks["hbm_gbs"], 4)
         else:
             entry["frac"] = round(tf / peaks["bf16_tflops_sustained"], 4)
             entry["frac_of_burst_peak"] = round(tf / peaks["bf16_tflops"], 4)
         programs[prog] = entry
     torch.cuda.synchronize()
-    extra_programs = {k: programs.pop(k) for k in wl.EXTRA_PROGRAMS}
+    extra_programs = {e[0]: programs.pop(e[0]) for e in extras}
     dominant = max(programs, key=lambda q: programs[q]["us_per_call"])
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
@@ -290,7 +295,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2: one step touches %d MB of distinct inputs" % (in_bytes // 1000000),
                    "seed": rank, "parallelism": f"replicas x{world} (no collective on the path)"},
         "clocks": clocks, "e2e": e2e,
-        "gpu_launches": args.steps * sum(KERNELS_PER_CALL.values()),
+        "gpu_launches": args.steps * sum(KERNELS_PER_CALL[q] for q in wl.PROGRAMS),   # kernels of the timed steps
         "roofline": roofline, "programs": programs, "extra_programs": extra_programs,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

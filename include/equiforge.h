@@ -103,6 +103,21 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O,
                         void* ws, size_t ws_bytes, void* stream);
 size_t ef_gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int L, int D);
 
+/* ---- Program 3b: decode attention with per-sequence key lengths -----------------------------
+ * The same rolling reducer over a batch whose sequences have different lengths (the serving
+ * case behind the decode workloads of Section 7.1, batch sizes 1/8/16): batch entry b attends
+ * keys [0, seq_lens[b]) of its K/V rows.  The chunks of all (batch, kv head) units still form
+ * one list cut into equal contiguous ranges (Section 6.1 thread-block mapping; Section 4.4
+ * Collection for units that span blocks), so a short sequence costs only its own bytes.
+ *   Q [B,Hq,D], K,V [B,Hkv,Lmax,D] (rows at and beyond seq_lens[b] are padding: never used,
+ *   may hold anything including NaN), seq_lens [B] int32 DEVICE pointer -> O [B,Hq,D].
+ *   seq_lens[b] is clamped to [0, Lmax]; an entry with no keys gets O[b] = 0.
+ * Supported: D == 128, Hq % Hkv == 0, Hq/Hkv <= 8, B <= 1024.
+ * Workspace: ef_gqa_decode_workspace_bytes(B, Hq, Hkv, Lmax, D). */
+ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, const void* seq_lens, void* O,
+                               int B, int Hq, int Hkv, int Lmax, int D, float scale,
+                               void* ws, size_t ws_bytes, void* stream);
+
 /* ---- Program 4: QK-normalised (causal) prefill attention ---------------------------------
  * qh = q * rsqrt(mean_d q^2 + eps) * gamma_q, kh likewise with gamma_k (over head_dim);
  * s_ij = scale * qh_i . kh_j for j <= i when causal != 0 (all j otherwise); softmax over j;

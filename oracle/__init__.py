@@ -83,6 +83,18 @@ def gqa_decode(Q, K, V, scale):
     return O
 
 
+def gqa_decode_varlen(Q, K, V, seq_lens, scale):
+    Q, pQ = _d(Q); K, pK = _d(K); V, pV = _d(V)
+    B, Hq, D = Q.shape; _, Hkv, L, _ = K.shape
+    assert K.shape == (B, Hkv, L, D) and V.shape == K.shape and Hq % Hkv == 0
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    assert lens.shape == (B,)
+    O = np.empty((B, Hq, D), dtype=np.float64)
+    _load().ef_oracle_gqa_decode_varlen(pQ, pK, pV, lens.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), _d(O)[1],
+                                        B, Hq, Hkv, L, D, ctypes.c_double(scale))
+    return O
+
+
 def qknorm_attn(Q, K, V, gamma_q, gamma_k, eps, scale, causal=1):
     Q, pQ = _d(Q); K, pK = _d(K); V, pV = _d(V)
     gamma_q, pgq = _d(gamma_q); gamma_k, pgk = _d(gamma_k)
@@ -114,6 +126,8 @@ def run(program: str, params: dict, tensors_f64: dict) -> np.ndarray:
         return rmsnorm_gated_mlp(t["X"], t["gamma"], t["Wgate"], t["Wup"], p["eps"])
     if program == "gqa_decode":
         return gqa_decode(t["Q"], t["K"], t["V"], p["scale"])
+    if program == "gqa_decode_varlen":
+        return gqa_decode_varlen(t["Q"], t["K"], t["V"], t["seq_lens"], p["scale"])
     if program == "qknorm_attn":
         return qknorm_attn(t["Q"], t["K"], t["V"], t["gamma_q"], t["gamma_k"], p["eps"], p["scale"], p.get("causal", 1))
     if program == "lora_linear":

@@ -159,6 +159,30 @@ void ef_oracle_gqa_decode(const double *Q, const double *K, const double *V, dou
     }
 }
 
+/* Program 3b (decode attention, per-sequence key lengths): batch entry b attends keys [0, len_b) of its
+ * K/V rows (len_b clamped to [0, L]); rows at and beyond len_b are padding and are never read.  An entry
+ * with no keys has no softmax; its output is defined as zero.  Otherwise exactly Program 3 per entry. */
+void ef_oracle_gqa_decode_varlen(const double *Q, const double *K, const double *V, const int *lens, double *O,
+                                 int B, int Hq, int Hkv, int L, int D, double scale) {
+    const int group = Hq / Hkv;
+#pragma omp parallel for schedule(static)
+    for (int bh = 0; bh < B * Hq; ++bh) {
+        const int b = bh / Hq, h = bh % Hq, g = h / group;
+        int len = lens[b];
+        if (len < 0) len = 0;
+        if (len > L) len = L;
+        double *out = O + (size_t)bh * D;
+        if (len == 0) {
+            for (int d = 0; d < D; ++d) out[d] = 0.0;
+            continue;
+        }
+        double *s = (double *)malloc((size_t)len * sizeof(double));
+        const size_t kv_off = ((size_t)b * Hkv + g) * (size_t)L * D;
+        attend_row(Q + (size_t)bh * D, K + kv_off, V + kv_off, (size_t)D, len, D, scale, s, out);
+        free(s);
+    }
+}
+
 /* Program 4 (prefill attention with RMS-normalised queries and keys):
  *   qh_i = q_i * inv_rms(q_i) * gamma_q;  kh_j = k_j * inv_rms(k_j) * gamma_k  (over head_dim),
  *   then vanilla attention (M0) per (b,h), row i attending keys j <= i when causal.

@@ -19,7 +19,8 @@ EXPORTS = [
     "ef_rmsnorm_matmul", "ef_rmsnorm_matmul_workspace_bytes",
     "ef_gated_mlp", "ef_gated_mlp_workspace_bytes",
     "ef_rmsnorm_gated_mlp", "ef_rmsnorm_gated_mlp_workspace_bytes",
-    "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_static", "ef_gqa_decode_static_max_units",
+    "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_varlen", "ef_gqa_decode_static",
+    "ef_gqa_decode_static_max_units",
     "ef_qknorm_attn", "ef_qknorm_attn_workspace_bytes",
     "ef_lora_linear", "ef_lora_linear_workspace_bytes",
     "ef_workspace_init", "ef_check_status", "ef_status_string", "ef_last_cuda_error", "ef_version",
@@ -49,6 +50,7 @@ def lib():
         L.ef_rmsnorm_gated_mlp_workspace_bytes.argtypes = [i, i, i]
         L.ef_gqa_decode.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
         L.ef_gqa_decode_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.ef_gqa_decode_varlen.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
         L.ef_gqa_decode_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp]
         L.ef_gqa_decode_static_max_units.argtypes = []
         L.ef_qknorm_attn.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, f, f, i, vp, sz, vp]
@@ -182,6 +184,22 @@ def gqa_decode(Q, K, V, scale, ws: Workspace, out=None):
     return O
 
 
+def gqa_decode_varlen(Q, K, V, seq_lens, scale, ws: Workspace, out=None):
+    """Decode attention where batch entry b attends keys [0, seq_lens[b]); seq_lens is a CUDA int32 tensor [B]."""
+    import torch
+
+    B, Hq, D = Q.shape
+    _, Hkv, L, _ = K.shape
+    if seq_lens.dtype != torch.int32 or not seq_lens.is_cuda or not seq_lens.is_contiguous() or seq_lens.numel() != B:
+        raise ValueError("seq_lens must be a contiguous CUDA int32 tensor with one entry per batch element")
+    O = out if out is not None else torch.empty((B, Hq, D), dtype=torch.bfloat16, device=Q.device)
+    wp, wb = _ws_args(ws, gqa_decode_workspace_bytes(B, Hq, Hkv, L, D), "ef_gqa_decode_varlen")
+    _check(lib().ef_gqa_decode_varlen(_ptr(Q, "Q"), _ptr(K, "K"), _ptr(V, "V"), ctypes.c_void_p(seq_lens.data_ptr()),
+                                      _ptr(O, "O"), B, Hq, Hkv, L, D, float(scale), wp, wb, _stream()),
+           "ef_gqa_decode_varlen")
+    return O
+
+
 def gqa_decode_static(Q, K, V, scale, out=None):
     """Decode attention through ef_gqa_decode_static: no workspace argument, nothing allocated by
     the call itself (the output tensor is the caller's: pass `out` to avoid torch allocating one).
@@ -229,7 +247,7 @@ def workspace_bytes(program: str, p: dict) -> int:
         return gated_mlp_workspace_bytes(p["M"], p["K"], p["N"])
     if program == "rmsnorm_gated_mlp":
         return rmsnorm_gated_mlp_workspace_bytes(p["M"], p["K"], p["N"])
-    if program == "gqa_decode":
+    if program in ("gqa_decode", "gqa_decode_varlen"):
         return gqa_decode_workspace_bytes(p["B"], p["Hq"], p["Hkv"], p["L"], p["D"])
     if program == "qknorm_attn":
         return qknorm_attn_workspace_bytes(p["B"], p["H"], p["S"], p["D"])
@@ -248,6 +266,8 @@ def run(program: str, p: dict, t: dict, ws: Workspace, out=None):
         return rmsnorm_gated_mlp(t["X"], t["gamma"], t["Wgate"], t["Wup"], p["eps"], ws, out)
     if program == "gqa_decode":
         return gqa_decode(t["Q"], t["K"], t["V"], p["scale"], ws, out)
+    if program == "gqa_decode_varlen":
+        return gqa_decode_varlen(t["Q"], t["K"], t["V"], t["seq_lens"], p["scale"], ws, out)
     if program == "qknorm_attn":
         return qknorm_attn(t["Q"], t["K"], t["V"], t["gamma_q"], t["gamma_k"], p["eps"], p["scale"],
                            p.get("causal", 1), ws, out)

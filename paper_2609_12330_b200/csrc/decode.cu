@@ -39,13 +39,16 @@ constexpr int kSlotFloats = kMaxGroup * kRowFloats;
 constexpr int kMergeBytes = kConsumerWarps * kSlotFloats * 4;
 constexpr int kMaxGrid = 256;                     // upper bound on the persistent grid
 constexpr int kBarBytes = 128 + kMaxGrid * 4;     // barriers, flags, slot table of the final merge
-constexpr int kSmemBytes = 1024 /*align slack*/ + kStages * kStageBytes + kMergeBytes + kBarBytes;
+constexpr int kMaxVarlenB = 1024;                 // batch entries of the per-sequence-length variant
+constexpr int kCumBytes = (2 * kMaxVarlenB + 4) * 4;   // chunk-count prefix over the batch, base/rem, clamped lengths (that variant only)
+constexpr int kSmemBytes = 1024 /*align slack*/ + kStages * kStageBytes + kMergeBytes + kBarBytes + kCumBytes;
 
 struct Params {
     const __nv_bfloat16* Q;
     __nv_bfloat16* O;
     int B, Hq, Hkv, L, G;
-    int n_chunks;      // chunks per (b, kv head) unit
+    const int* seq_lens;   // per-sequence-length variant: keys [0, seq_lens[b]) of batch entry b are attended
+    int n_chunks;      // chunks per (b, kv head) unit (uniform variant)
     int total_items;   // units * n_chunks  (< 2^30)
     int base, rem;     // block c owns base + (c < rem) consecutive items
     float scale_log2;  // scale * log2(e)
@@ -68,11 +71,51 @@ __device__ __forceinline__ int owner_of(int x, int base, int rem) {
     const int big = rem * (base + 1);
     return x < big ? x / (base + 1) : rem + (x - big) / base;
 }
+// Where item x of the flattened chunk list lies.  Uniform lengths: every (batch, kv head) unit has n_chunks chunks.
+// Per-sequence lengths: batch entry b has nb_b = ceil(len_b / 128) chunks per unit, cum[b] = sum of nb over
+// earlier entries, and its Hkv units follow each other, so entry b owns items [Hkv*cum[b], Hkv*cum[b+1]).
+// Layout of `cum` (shared memory, per-sequence-length variant only): [0..B] prefix, [B+1] base, [B+2] rem,
+// [B+3 ..] clamped lengths.
+struct Where {
+    int unit;         // b * Hkv + kv head
+    int chunk;        // chunk of x within the unit
+    int unit_begin;   // item index of the unit's first chunk
+    int n_chunks;     // chunks of the unit
+    int len;          // keys of the unit
+};
+template <bool VARLEN>
+__device__ __forceinline__ Where locate(int x, const Params& p, const int* cum) {
+    Where w;
+    if (!VARLEN) {
+        w.unit = x / p.n_chunks;
+        w.unit_begin = w.unit * p.n_chunks;
+        w.chunk = x - w.unit_begin;
+        w.n_chunks = p.n_chunks;
+        w.len = p.L;
+    } else {
+        int lo = 0, hi = p.B;   // largest b with Hkv * cum[b] <= x (entries without keys own no items)
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (p.Hkv * cum[mid] <= x) lo = mid; else hi = mid;
+        }
+        const int nb = cum[lo + 1] - cum[lo];
+        const int rel = x - p.Hkv * cum[lo];
+        const int kvh = rel / nb;
+        w.unit = lo * p.Hkv + kvh;
+        w.chunk = rel - kvh * nb;
+        w.unit_begin = x - w.chunk;
+        w.n_chunks = nb;
+        w.len = cum[p.B + 3 + lo];   // clamped length, cached by the prologue
+    }
+    return w;
+}
 // Partial-state slot of block c for `unit`: 0 if the unit is the first one the block touches, else 1.
-__device__ __forceinline__ int slot_of(int c, int unit, int base, int rem, int n_chunks) {
-    return 2 * c + ((range_begin(c, base, rem) / n_chunks) == unit ? 0 : 1);
+template <bool VARLEN>
+__device__ __forceinline__ int slot_of(int c, int unit, int base, int rem, const Params& p, const int* cum) {
+    return 2 * c + (locate<VARLEN>(range_begin(c, base, rem), p, cum).unit == unit ? 0 : 1);
 }
 
+template <bool VARLEN>
 __global__ void __launch_bounds__(kThreads, 1)
 gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
     extern __shared__ uint8_t smem_raw[];
@@ -86,12 +129,11 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 3 * kStages);
     uint32_t* is_last = const_cast<uint32_t*>(abort_flag) + 1;
     int* slot_table = reinterpret_cast<int*>(bars) + 32;  // [kMaxGrid]
+    int* cum = reinterpret_cast<int*>(smem + kStages * kStageBytes + kMergeBytes + kBarBytes);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-    const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
-    const int it_end = range_begin(blockIdx.x + 1, p.base, p.rem);
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -107,6 +149,60 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     __syncthreads();
     pdl_wait();  // everything below may touch global memory of the previous kernel in the stream
 
+    int base = p.base, rem = p.rem;
+    if (VARLEN) {
+        // Every block builds the same chunk-count prefix over the batch (warp 0: a serial piece per lane, then a
+        // shuffle scan of the lane totals) and derives the partition of the item list from its total.
+        if (warp == 0) {
+            const int per = (p.B + 31) / 32;
+            const int b0 = lane * per;
+            int sum = 0;
+            for (int i = 0; i < per; ++i) {
+                const int b = b0 + i;
+                if (b < p.B) {
+                    int len = p.seq_lens[b];
+                    len = len < 0 ? 0 : (len > p.L ? p.L : len);
+                    cum[p.B + 3 + b] = len;
+                    sum += (len + kChunk - 1) / kChunk;
+                }
+            }
+            int incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            int run = incl - sum;   // chunks of the entries before this lane's piece
+            for (int i = 0; i < per; ++i) {
+                const int b = b0 + i;
+                if (b < p.B) {
+                    cum[b] = run;
+                    run += (cum[p.B + 3 + b] + kChunk - 1) / kChunk;
+                }
+            }
+            if (lane == 31) {
+                cum[p.B] = incl;
+                const int total = incl * p.Hkv;
+                cum[p.B + 1] = total / static_cast<int>(gridDim.x);
+                cum[p.B + 2] = total % static_cast<int>(gridDim.x);
+            }
+        }
+        __syncthreads();
+        base = cum[p.B + 1];
+        rem = cum[p.B + 2];
+        // entries without keys: softmax over nothing, the output row is defined as zero (block 0 writes it)
+        if (blockIdx.x == 0) {
+            for (int b = 0; b < p.B; ++b) {
+                if (cum[b + 1] == cum[b]) {
+                    for (int i = tid; i < p.Hq * (kD / 8); i += kThreads)
+                        reinterpret_cast<uint4*>(p.O + static_cast<size_t>(b) * p.Hq * kD)[i] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+        }
+    }
+    const int it_begin = range_begin(blockIdx.x, base, rem);
+    const int it_end = range_begin(blockIdx.x + 1, base, rem);
+
     if (warp == kConsumerWarps) {
         // ------------------------------ producer warp ------------------------------
         if (lane == 0) {
@@ -114,8 +210,9 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             tma_prefetch_desc(&tmV);
             int stage = 0;
             uint32_t phase = 0;
-            int unit = it_begin / p.n_chunks;
-            int chunk = it_begin - unit * p.n_chunks;
+            Where w = {0, 0, 0, 1, 0};
+            if (it_begin < it_end) w = locate<VARLEN>(it_begin, p, cum);
+            int unit = w.unit, chunk = w.chunk, unit_chunks = w.n_chunks;
             for (int it = it_begin; it < it_end; ++it) {
                 if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) break;
                 uint8_t* st = stages + stage * kStageBytes;
@@ -127,7 +224,15 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 tma_load_3d(st + 2 * kHalfBytes, &tmV, &fullV[stage], 0, key0, unit);
                 tma_load_3d(st + 3 * kHalfBytes, &tmV, &fullV[stage], 64, key0, unit);
                 if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                if (++chunk == p.n_chunks) { chunk = 0; ++unit; }
+                if (++chunk == unit_chunks) {
+                    chunk = 0;
+                    ++unit;
+                    if (VARLEN && it + 1 < it_end) {   // the next unit may belong to another batch entry
+                        const Where nx = locate<VARLEN>(it + 1, p, cum);
+                        unit = nx.unit;
+                        unit_chunks = nx.n_chunks;
+                    }
+                }
             }
         }
     } else {
@@ -139,9 +244,11 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         int it = it_begin;
         bool ok = true;
         while (it < it_end && ok) {
-            const int unit = it / p.n_chunks;
-            const int c0 = it - unit * p.n_chunks;
-            const int unit_end = (unit + 1) * p.n_chunks;
+            const Where w = locate<VARLEN>(it, p, cum);
+            const int unit = w.unit;
+            const int c0 = w.chunk;
+            const int unit_end = w.unit_begin + w.n_chunks;
+            const int len = w.len;   // keys of this unit
             const int seg_end = unit_end < it_end ? unit_end : it_end;
             const int n_seg = seg_end - it;
             const bool whole_unit = (c0 == 0) && (seg_end == unit_end);
@@ -193,8 +300,8 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll
                 for (int nt = 0; nt < 4; ++nt) {
                     const int key = key_base + nt * 8 + 2 * t4;
-                    s[nt][0] = (key < p.L) ? s[nt][0] * p.scale_log2 : -INFINITY;
-                    s[nt][1] = (key + 1 < p.L) ? s[nt][1] * p.scale_log2 : -INFINITY;
+                    s[nt][0] = (key < len) ? s[nt][0] * p.scale_log2 : -INFINITY;
+                    s[nt][1] = (key + 1 < len) ? s[nt][1] * p.scale_log2 : -INFINITY;
                     mx = fmaxf(mx, fmaxf(s[nt][0], s[nt][1]));
                 }
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -217,6 +324,21 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 for (int i = 0; i < 16; ++i) { o[i][0] *= resc; o[i][1] *= resc; }
                 // ---- value += P V for this warp's 32 keys: 2 k-steps x 16 n-tiles
                 if (!warp_wait(&fullV[stage], phase, abort_flag, p.status, 3)) { ok = false; break; }
+                if (VARLEN && (c0 + ch + 1) * kChunk > len) {
+                    // Keys at and beyond the sequence length are padding that may hold anything (their weight
+                    // is 0, but 0 * NaN is NaN): this warp zeroes its own padded V rows before reading them.
+                    const int key_l = warp * kKeysPerWarp + lane;   // one row per lane
+                    if ((c0 + ch) * kChunk + key_l >= len) {
+                        uint8_t* vrow = stages + stage * kStageBytes + 2 * kHalfBytes + key_l * 128;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            *reinterpret_cast<uint4*>(vrow + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+                            *reinterpret_cast<uint4*>(vrow + kHalfBytes + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+                    fence_proxy_async_smem();   // the stage is refilled by the async proxy later
+                    __syncwarp();
+                }
 #pragma unroll
                 for (int kk = 0; kk < 2; ++kk) {
                     const int key_local = warp * kKeysPerWarp + kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
@@ -247,7 +369,7 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 for (int i = 0; i < 16; ++i) *reinterpret_cast<float2*>(row + i * 8 + 2 * t4) = make_float2(o[i][0], o[i][1]);
             }
             consumer_sync();
-            float* pslot = p.partials + static_cast<size_t>(slot_of(blockIdx.x, unit, p.base, p.rem, p.n_chunks)) * kSlotFloats;
+            float* pslot = p.partials + static_cast<size_t>(slot_of<VARLEN>(blockIdx.x, unit, base, rem, p, cum)) * kSlotFloats;
             for (int idx = tid; idx < p.G * kD; idx += kConsumerThreads) {
                 const int r = idx >> 7, d = idx & (kD - 1);
                 float mw[kConsumerWarps];
@@ -275,15 +397,15 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 // Collection + parallel reduce across blocks: the block that arrives last merges.
                 __threadfence();
                 consumer_sync();
-                const int c_first = owner_of(unit * p.n_chunks, p.base, p.rem);
-                const int c_last = owner_of(unit_end - 1, p.base, p.rem);
+                const int c_first = owner_of(w.unit_begin, base, rem);
+                const int c_last = owner_of(unit_end - 1, base, rem);
                 const int n_parts = c_last - c_first + 1;
                 if (tid == 0) {
                     const uint32_t prev = atomicAdd(&p.counters[unit], 1u);
                     *is_last = (prev == static_cast<uint32_t>(n_parts - 1)) ? 1u : 0u;
                 }
                 for (int i = tid; i < n_parts; i += kConsumerThreads)
-                    slot_table[i] = slot_of(c_first + i, unit, p.base, p.rem, p.n_chunks);
+                    slot_table[i] = slot_of<VARLEN>(c_first + i, unit, base, rem, p, cum);
                 consumer_sync();
                 if (*is_last) {
                     __threadfence();
@@ -363,7 +485,7 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
 
     static bool attr_set[64] = {};
     if (!attr_set[di.device]) {
-        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            decode::kSmemBytes));
         attr_set[di.device] = true;
     }
@@ -371,6 +493,7 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
     p.Q = static_cast<const __nv_bfloat16*>(Q);
     p.O = static_cast<__nv_bfloat16*>(O);
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.L = L; p.G = Hq / Hkv;
+    p.seq_lens = nullptr;
     p.n_chunks = static_cast<int>(n_chunks);
     p.total_items = static_cast<int>(n_chunks * static_cast<long long>(n_units));
     int grid = di.num_sms < p.total_items ? di.num_sms : p.total_items;
@@ -382,7 +505,62 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
     p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
-    EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
+    EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<false>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
+                             static_cast<cudaStream_t>(stream), tmK, tmV, p));
+    return EF_OK;
+}
+
+ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, const void* seq_lens, void* O, int B, int Hq,
+                               int Hkv, int Lmax, int D, float scale, void* ws, size_t ws_bytes, void* stream) {
+    using namespace ef;
+    if (!Q || !K || !V || !O || !seq_lens) return EF_ERR_NULL;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Lmax <= 0 || D <= 0 || Hq % Hkv != 0) return EF_ERR_SHAPE;
+    if (D != decode::kD || Hq / Hkv > decode::kMaxGroup || B > decode::kMaxVarlenB) return EF_ERR_UNSUPPORTED;
+    const size_t n_units = static_cast<size_t>(B) * Hkv;
+    const size_t counters_bytes = (n_units * sizeof(uint32_t) + 255) & ~size_t(255);
+    if (kHeaderBytes + counters_bytes > 65536) return EF_ERR_UNSUPPORTED;  // counters must lie in the init window
+    const long long n_chunks = (static_cast<long long>(Lmax) + decode::kChunk - 1) / decode::kChunk;
+    if (n_chunks * static_cast<long long>(n_units) >= (1LL << 30)) return EF_ERR_UNSUPPORTED;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(seq_lens, 4)) return EF_ERR_ALIGN;
+    if (!ws || ws_bytes < ef_gqa_decode_workspace_bytes(B, Hq, Hkv, Lmax, D)) return EF_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return EF_ERR_ALIGN;
+    DeviceInfo di;
+    if (!current_device_info(&di)) return EF_ERR_CUDA;
+    if (di.cc_major != 10) return EF_ERR_ARCH;
+
+    CUtensorMap tmK, tmV;
+    const uint64_t dims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Lmax), n_units};
+    const uint64_t strides[2] = {static_cast<uint64_t>(D) * 2, static_cast<uint64_t>(Lmax) * D * 2};
+    const uint32_t box[3] = {64, decode::kChunk, 1};
+    ef_status st = encode_tmap_bf16(&tmK, K, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != EF_OK) return st;
+    st = encode_tmap_bf16(&tmV, V, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != EF_OK) return st;
+
+    static bool attr_set[64] = {};
+    if (!attr_set[di.device]) {
+        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           decode::kSmemBytes));
+        attr_set[di.device] = true;
+    }
+    decode::Params p;
+    p.Q = static_cast<const __nv_bfloat16*>(Q);
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.L = Lmax; p.G = Hq / Hkv;
+    p.seq_lens = static_cast<const int*>(seq_lens);
+    p.n_chunks = static_cast<int>(n_chunks);
+    p.total_items = 0;   // the lengths live on the device: every block derives the item list and its range itself
+    p.base = 0;
+    p.rem = 0;
+    const long long max_items = n_chunks * static_cast<long long>(n_units);
+    int grid = di.num_sms < max_items ? di.num_sms : static_cast<int>(max_items);
+    if (grid > decode::kMaxGrid) grid = decode::kMaxGrid;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    p.status = reinterpret_cast<uint32_t*>(w);
+    p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
+    p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
+    EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<true>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
                              static_cast<cudaStream_t>(stream), tmK, tmV, p));
     return EF_OK;
 }

@@ -12,9 +12,9 @@ def run_parity(program, seed=0, size="small", check_repeat=True, oracle_fn=None,
     import paper_2609_12330_b200 as ef
 
     p, t = wl.make_inputs(program, seed=seed, size=size, **over)
-    f64 = {k: wl.bf16_bits_to_f64(v) for k, v in t.items()}
+    f64 = {k: wl.to_f64(k, v) for k, v in t.items()}
     ref = oracle.run(program, p, f64) if oracle_fn is None else oracle_fn(p, f64)
-    dev = {k: wl.bf16_bits_to_torch(v, "cuda") for k, v in t.items()}
+    dev = {k: wl.to_torch(k, v, "cuda") for k, v in t.items()}
     ws = ef.Workspace(ef.workspace_bytes(program, p))
     out = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
     ef.run(program, p, dev, ws, out=out)

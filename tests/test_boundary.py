@@ -55,6 +55,12 @@ def test_host_side_argument_validation(lib):
     # workspace
     assert lib.ef_gqa_decode(one, one, one, one, 1, 4, 1, 8, 128, 1.0, null, 0, null) == 5
     assert lib.ef_gqa_decode(one, one, one, one, 1, 4, 1, 8, 128, 1.0, one, 16, null) == 5
+    # the per-sequence-length decode: same rules, plus the length array and the batch limit
+    assert lib.ef_gqa_decode_varlen(one, one, one, null, one, 1, 4, 1, 8, 128, 1.0, one, 1 << 30, null) == 1
+    assert lib.ef_gqa_decode_varlen(one, one, one, one, one, 1, 5, 2, 8, 128, 1.0, one, 1 << 30, null) == 2
+    assert lib.ef_gqa_decode_varlen(one, one, one, one, one, 1025, 4, 1, 8, 128, 1.0, one, 1 << 30, null) == 3   # B > 1024
+    assert lib.ef_gqa_decode_varlen(one, one, one, p(4098), one, 1, 4, 1, 8, 128, 1.0, one, 1 << 30, null) == 4
+    assert lib.ef_gqa_decode_varlen(one, one, one, one, one, 1, 4, 1, 8, 128, 1.0, one, 16, null) == 5
     assert lib.ef_workspace_init(null, 4096, null) == 1
     assert lib.ef_workspace_init(one, 16, null) == 5
 

@@ -274,6 +274,40 @@ def test_decode_against_scipy_softmax_and_head_mapping():
     np.testing.assert_allclose(oracle.gqa_decode(Q, K[:, :, perm], V[:, :, perm], scale), o, **TOL)
 
 
+def test_decode_varlen_against_scipy_softmax_per_entry():
+    """Per-sequence lengths: entry b is plain softmax attention over its first len_b keys (library routines on the
+    truncated tensors), padding rows are never read (NaN there changes nothing), an entry without keys is zero,
+    lengths are clamped to [0, L], and a length-1 entry returns v_0."""
+    B, Hq, Hkv, L, D = 5, 4, 2, 9, 3
+    Q = RNG.standard_normal((B, Hq, D)); K = RNG.standard_normal((B, Hkv, L, D)); V = RNG.standard_normal((B, Hkv, L, D))
+    lens = np.array([9, 1, 0, 4, 7], dtype=np.int32)
+    scale = 0.41
+    Kp, Vp = K.copy(), V.copy()
+    for b in range(B):
+        Kp[b, :, lens[b]:] = np.nan
+        Vp[b, :, lens[b]:] = np.nan
+    o = oracle.gqa_decode_varlen(Q, Kp, Vp, lens, scale)
+    assert np.all(np.isfinite(o))
+    for b in range(B):
+        n = lens[b]
+        if n == 0:
+            assert np.array_equal(o[b], np.zeros((Hq, D)))
+            continue
+        Kx, Vx = np.repeat(K[b, :, :n], Hq // Hkv, axis=0), np.repeat(V[b, :, :n], Hq // Hkv, axis=0)
+        ref = np.einsum("hl,hld->hd", softmax(np.einsum("hd,hld->hl", Q[b], Kx) * scale, axis=-1), Vx)
+        np.testing.assert_allclose(o[b], ref, **TOL)
+    for h in range(Hq):
+        assert np.array_equal(o[1, h], V[1, h // 2, 0])           # one key: the output is that key's value row
+    # all lengths equal to L: the uniform program, bit for bit (same routine on the same rows)
+    full = np.full(B, L, dtype=np.int32)
+    assert np.array_equal(oracle.gqa_decode_varlen(Q, K, V, full, scale), oracle.gqa_decode(Q, K, V, scale))
+    # clamping: a length beyond L means L, a negative one means 0
+    odd = np.array([L + 50, -2, 3, L, 0], dtype=np.int32)
+    oc = oracle.gqa_decode_varlen(Q, K, V, odd, scale)
+    ok = oracle.gqa_decode_varlen(Q, K, V, np.array([L, 0, 3, L, 0], dtype=np.int32), scale)
+    assert np.array_equal(oc, ok)
+
+
 def test_decode_max_shift_invariance():
     # adding u to every key with q.u = c shifts every logit by c*scale; softmax is invariant
     # (the basis of the repair h(c,s,s') = c*exp(s-s'), Section 4.2)

@@ -22,7 +22,7 @@ import numpy as np
 
 PROGRAMS = ("rmsnorm_matmul", "gated_mlp", "gqa_decode", "qknorm_attn", "lora_linear")
 # programs beyond the five benchmark configurations (the "next" rows of the scope table)
-EXTRA_PROGRAMS = ("rmsnorm_gated_mlp",)
+EXTRA_PROGRAMS = ("rmsnorm_gated_mlp", "gqa_decode_varlen")
 _PROGRAM_ID = {name: i for i, name in enumerate(PROGRAMS + EXTRA_PROGRAMS)}
 
 
@@ -48,6 +48,25 @@ def bf16_bits_to_torch(bits: np.ndarray, device="cpu"):
 
     t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16).copy())
     return t.view(torch.bfloat16).to(device)
+
+
+INT_TENSORS = ("seq_lens",)   # tensor names that are int32, not bf16 bit patterns
+
+
+def to_torch(name: str, arr: np.ndarray, device="cpu"):
+    """Torch tensor for one entry of make_inputs()'s tensor dict (bf16 bits, or int32 for INT_TENSORS)."""
+    if name in INT_TENSORS:
+        import torch
+
+        return torch.from_numpy(np.ascontiguousarray(arr, dtype=np.int32).copy()).to(device)
+    return bf16_bits_to_torch(arr, device)
+
+
+def to_f64(name: str, arr: np.ndarray) -> np.ndarray:
+    """Oracle-side view of one entry of the tensor dict (exact widening; int tensors stay int32)."""
+    if name in INT_TENSORS:
+        return np.ascontiguousarray(arr, dtype=np.int32)
+    return bf16_bits_to_f64(arr)
 
 
 def torch_bf16_to_f64(t) -> np.ndarray:
@@ -91,6 +110,10 @@ SHAPES = {
     "gqa_decode": {
         "full": dict(B=8, Hq=32, Hkv=8, L=4096, D=128, scale=1.0 / np.sqrt(128.0)),
         "small": dict(B=2, Hq=8, Hkv=2, L=333, D=128, scale=1.0 / np.sqrt(128.0)),
+    },
+    "gqa_decode_varlen": {  # serving batch with a length mix: lengths uniform in [1, L], one full, one of length 1
+        "full": dict(B=16, Hq=32, Hkv=8, L=4096, D=128, scale=1.0 / np.sqrt(128.0)),
+        "small": dict(B=5, Hq=8, Hkv=2, L=333, D=128, scale=1.0 / np.sqrt(128.0)),
     },
     "qknorm_attn": {
         "full": dict(B=2, H=32, S=2048, D=128, eps=1e-6, scale=1.0 / np.sqrt(128.0), causal=1),
@@ -138,6 +161,26 @@ def make_inputs(program: str, seed: int = 0, size: str = "full", **overrides):
             "K": g(1, (B, Hkv, L, D), 0.0, 1.0),
             "V": g(2, (B, Hkv, L, D), 0.0, 1.0),
         }
+    elif program == "gqa_decode_varlen":
+        B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
+        lens = p.pop("lens", None)
+        pad_nan = p.pop("pad_nan", True)
+        if lens is None:
+            ss = np.random.SeedSequence([int(seed), _PROGRAM_ID[program], 99])
+            lens = np.random.Generator(np.random.Philox(ss)).integers(1, L + 1, size=B)
+            lens[0] = L
+            if B > 1:
+                lens[1] = 1
+            if B > 2 and size == "small":
+                lens[2] = 0          # an entry without keys: its output is defined as zero
+        lens = np.asarray(lens, dtype=np.int32)
+        K, V = g(1, (B, Hkv, L, D), 0.0, 1.0), g(2, (B, Hkv, L, D), 0.0, 1.0)
+        for b in range(B if pad_nan else 0):   # padding rows hold NaN: neither side may let them reach the output
+            n = int(np.clip(lens[b], 0, L))
+            K[b, :, n:, :] = 0x7FC0
+            V[b, :, n:, :] = 0x7FC0
+        p["lens_sum"] = int(np.clip(lens, 0, L).sum())
+        t = {"Q": g(0, (B, Hq, D), 0.0, 1.0), "K": K, "V": V, "seq_lens": lens}
     elif program == "qknorm_attn":
         B, H, S, D = p["B"], p["H"], p["S"], p["D"]
         t = {
@@ -174,6 +217,10 @@ def algorithmic_work(program: str, p: dict) -> dict:
     if program == "gqa_decode":
         B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
         return dict(flops=4 * B * Hq * L * D, bytes=2 * (2 * B * Hkv * L * D + 2 * B * Hq * D))
+    if program == "gqa_decode_varlen":   # needs the lengths: p["lens_sum"] = sum of clamped lengths
+        Hq, Hkv, D = p["Hq"], p["Hkv"], p["D"]
+        tot = int(p["lens_sum"])
+        return dict(flops=4 * Hq * tot * D, bytes=2 * (2 * Hkv * tot * D + 2 * p["B"] * Hq * D))
     if program == "qknorm_attn":
         B, H, S, D = p["B"], p["H"], p["S"], p["D"]
         pairs = S * (S + 1) // 2 if p.get("causal", 1) else S * S

@@ -89,6 +89,21 @@ ef_status ef_rmsnorm_gated_mlp(const void* X, const void* gamma, const void* Wga
                                void* ws, size_t ws_bytes, void* stream);
 size_t ef_rmsnorm_gated_mlp_workspace_bytes(int M, int K, int N);
 
+/* ---- LayerNorm fused into a projection --------------------------------------------------------
+ * Y = LayerNorm(X) @ W,  LayerNorm(x)_k = (x_k - mean) * rsqrt(var + eps) * gamma_k + beta_k with
+ * mean and (biased) variance over the row (the paper names the LayerNorm+GEMM workload without
+ * defining it, Sections 7.1 and 7.2: this is the standard operator).  The mean subtraction does not
+ * commute with the contraction as a row scale, so the operand staged in shared memory is
+ * (x - mean) * gamma; the inverse standard deviation is invariant along K and scales the finished
+ * projection (Table 1, factor motion); beta @ W is produced by the same MMA from a spare operand
+ * row.  One kernel.
+ *   X [M,K], gamma [K], beta [K], W [K,N] -> Y [M,N].
+ * Supported: M <= 15, K % 64 == 0, K <= 4096, N % 8 == 0. */
+ef_status ef_layernorm_matmul(const void* X, const void* gamma, const void* beta, const void* W, void* Y,
+                              int M, int K, int N, float eps,
+                              void* ws, size_t ws_bytes, void* stream);
+size_t ef_layernorm_matmul_workspace_bytes(int M, int K, int N);
+
 /* ---- Program 3: grouped-query decode attention -------------------------------------------
  * One query token per sequence attends all L cached keys: for query head h and kv head
  * g = h / (Hq/Hkv):  O[b,h] = softmax_j(scale * Q[b,h] . K[b,g,j]) @ V[b,g].

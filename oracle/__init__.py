@@ -56,6 +56,15 @@ def rmsnorm_matmul(X, gamma, W, eps):
     return Y
 
 
+def layernorm_matmul(X, gamma, beta, W, eps):
+    X, pX = _d(X); gamma, pg = _d(gamma); beta, pb = _d(beta); W, pW = _d(W)
+    M, K = X.shape; N = W.shape[1]
+    assert W.shape[0] == K and gamma.shape == (K,) and beta.shape == (K,)
+    Y = np.empty((M, N), dtype=np.float64)
+    _load().ef_oracle_layernorm_matmul(pX, pg, pb, pW, _d(Y)[1], M, K, N, ctypes.c_double(eps))
+    return Y
+
+
 def gated_mlp(X, Wgate, Wup):
     X, pX = _d(X); Wgate, pG = _d(Wgate); Wup, pU = _d(Wup)
     M, K = X.shape; N = Wgate.shape[1]
@@ -120,6 +129,8 @@ def run(program: str, params: dict, tensors_f64: dict) -> np.ndarray:
     t, p = tensors_f64, params
     if program == "rmsnorm_matmul":
         return rmsnorm_matmul(t["X"], t["gamma"], t["W"], p["eps"])
+    if program == "layernorm_matmul":
+        return layernorm_matmul(t["X"], t["gamma"], t["beta"], t["W"], p["eps"])
     if program == "gated_mlp":
         return gated_mlp(t["X"], t["Wgate"], t["Wup"])
     if program == "rmsnorm_gated_mlp":

@@ -69,6 +69,29 @@ void ef_oracle_rmsnorm_matmul(const double *X, const double *gamma, const double
     }
 }
 
+/* LayerNorm followed by a projection (the LayerNorm+GEMM workload, Sections 7.1 and 7.2; the paper does not
+ * define the operator: standard LayerNorm, biased variance, eps inside the square root):
+ *   mu_i = mean_k x_ik;  var_i = mean_k (x_ik - mu_i)^2;  xn_ik = (x_ik - mu_i) / sqrt(var_i + eps) * gamma_k + beta_k;
+ *   Y = xn @ W.   X [M,K], gamma [K], beta [K], W [K,N] -> Y [M,N]. */
+void ef_oracle_layernorm_matmul(const double *X, const double *gamma, const double *beta, const double *W, double *Y,
+                                int M, int K, int N, double eps) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < M; ++i) {
+        double *xn = (double *)malloc((size_t)K * sizeof(double));
+        const double *x = X + (size_t)i * K;
+        double mu = 0.0;
+        for (int k = 0; k < K; ++k) mu += x[k];
+        mu /= (double)K;
+        double var = 0.0;
+        for (int k = 0; k < K; ++k) var += (x[k] - mu) * (x[k] - mu);
+        var /= (double)K;
+        const double r = 1.0 / sqrt(var + eps);
+        for (int k = 0; k < K; ++k) xn[k] = (x[k] - mu) * r * gamma[k] + beta[k];
+        row_times_matrix(xn, W, Y + (size_t)i * N, K, N);
+        free(xn);
+    }
+}
+
 /* SiLU(z) = z * sigmoid(z), evaluated without overflow for either sign. */
 static double silu(double z) {
     if (z >= 0.0) return z / (1.0 + exp(-z));

@@ -19,6 +19,7 @@ EXPORTS = [
     "ef_rmsnorm_matmul", "ef_rmsnorm_matmul_workspace_bytes",
     "ef_gated_mlp", "ef_gated_mlp_workspace_bytes",
     "ef_rmsnorm_gated_mlp", "ef_rmsnorm_gated_mlp_workspace_bytes",
+    "ef_layernorm_matmul", "ef_layernorm_matmul_workspace_bytes",
     "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_varlen", "ef_gqa_decode_static",
     "ef_gqa_decode_static_max_units",
     "ef_qknorm_attn", "ef_qknorm_attn_workspace_bytes",
@@ -48,6 +49,8 @@ def lib():
         L.ef_gated_mlp_workspace_bytes.argtypes = [i, i, i]
         L.ef_rmsnorm_gated_mlp.argtypes = [vp, vp, vp, vp, vp, i, i, i, f, vp, sz, vp]
         L.ef_rmsnorm_gated_mlp_workspace_bytes.argtypes = [i, i, i]
+        L.ef_layernorm_matmul.argtypes = [vp, vp, vp, vp, vp, i, i, i, f, vp, sz, vp]
+        L.ef_layernorm_matmul_workspace_bytes.argtypes = [i, i, i]
         L.ef_gqa_decode.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
         L.ef_gqa_decode_workspace_bytes.argtypes = [i, i, i, i, i]
         L.ef_gqa_decode_varlen.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
@@ -124,6 +127,10 @@ def rmsnorm_gated_mlp_workspace_bytes(M, K, N):
     return int(lib().ef_rmsnorm_gated_mlp_workspace_bytes(M, K, N))
 
 
+def layernorm_matmul_workspace_bytes(M, K, N):
+    return int(lib().ef_layernorm_matmul_workspace_bytes(M, K, N))
+
+
 def gqa_decode_workspace_bytes(B, Hq, Hkv, L, D):
     return int(lib().ef_gqa_decode_workspace_bytes(B, Hq, Hkv, L, D))
 
@@ -169,6 +176,18 @@ def rmsnorm_gated_mlp(X, gamma, Wgate, Wup, eps, ws: Workspace, out=None):
     wp, wb = _ws_args(ws, rmsnorm_gated_mlp_workspace_bytes(M, K, N), "ef_rmsnorm_gated_mlp")
     _check(lib().ef_rmsnorm_gated_mlp(_ptr(X, "X"), _ptr(gamma, "gamma"), _ptr(Wgate, "Wgate"), _ptr(Wup, "Wup"),
                                       _ptr(Y, "Y"), M, K, N, float(eps), wp, wb, _stream()), "ef_rmsnorm_gated_mlp")
+    return Y
+
+
+def layernorm_matmul(X, gamma, beta, W, eps, ws: Workspace, out=None):
+    import torch
+
+    M, K = X.shape
+    N = W.shape[1]
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    wp, wb = _ws_args(ws, layernorm_matmul_workspace_bytes(M, K, N), "ef_layernorm_matmul")
+    _check(lib().ef_layernorm_matmul(_ptr(X, "X"), _ptr(gamma, "gamma"), _ptr(beta, "beta"), _ptr(W, "W"), _ptr(Y, "Y"),
+                                     M, K, N, float(eps), wp, wb, _stream()), "ef_layernorm_matmul")
     return Y
 
 
@@ -247,6 +266,8 @@ def workspace_bytes(program: str, p: dict) -> int:
         return gated_mlp_workspace_bytes(p["M"], p["K"], p["N"])
     if program == "rmsnorm_gated_mlp":
         return rmsnorm_gated_mlp_workspace_bytes(p["M"], p["K"], p["N"])
+    if program == "layernorm_matmul":
+        return layernorm_matmul_workspace_bytes(p["M"], p["K"], p["N"])
     if program in ("gqa_decode", "gqa_decode_varlen"):
         return gqa_decode_workspace_bytes(p["B"], p["Hq"], p["Hkv"], p["L"], p["D"])
     if program == "qknorm_attn":
@@ -264,6 +285,8 @@ def run(program: str, p: dict, t: dict, ws: Workspace, out=None):
         return gated_mlp(t["X"], t["Wgate"], t["Wup"], ws, out)
     if program == "rmsnorm_gated_mlp":
         return rmsnorm_gated_mlp(t["X"], t["gamma"], t["Wgate"], t["Wup"], p["eps"], ws, out)
+    if program == "layernorm_matmul":
+        return layernorm_matmul(t["X"], t["gamma"], t["beta"], t["W"], p["eps"], ws, out)
     if program == "gqa_decode":
         return gqa_decode(t["Q"], t["K"], t["V"], p["scale"], ws, out)
     if program == "gqa_decode_varlen":

@@ -36,6 +36,7 @@ constexpr int kMaxSmem = 227 * 1024;
 struct Params {
     const __nv_bfloat16* X;
     const __nv_bfloat16* gamma;  // NORM only
+    const __nv_bfloat16* beta;   // LayerNorm only
     __nv_bfloat16* Y;
     int M, K, N;
     int n_tiles, k_blocks, total_units;
@@ -58,8 +59,10 @@ __device__ __forceinline__ int slot_of(int c, int tile, int base, int rem, int k
 __device__ __forceinline__ float silu(float z) { return z / (1.f + __expf(-z)); }
 
 // NW = number of weight matrices sharing the X operand (1: RMSNorm+matmul, 2: gated MLP)
-// NORM = build the X operand as bf16(x * gamma) in shared memory and scale rows by r_m at the end
-template <int NW, bool NORM>
+// NORM = 1: build the X operand as bf16(x * gamma) in shared memory and scale rows by r_m at the end (RMSNorm);
+// NORM = 2: LayerNorm: the operand is bf16((x - mean) * gamma), r_m = rsqrt(var + eps), and one spare operand row
+//           holds beta, so the MMA itself produces beta @ W, which the epilogue adds unscaled
+template <int NW, int NORM>
 __global__ void __launch_bounds__(kThreads, 1)
 skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
               const __grid_constant__ CUtensorMap tmX, const Params p) {
@@ -82,9 +85,13 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
     float* rinv = reinterpret_cast<float*>(tmem_slot + 4);        // [16]
     int* slot_table = reinterpret_cast<int*>(tmem_slot + 4 + kMaxM);  // [kMaxGrid]
     float* ssw = reinterpret_cast<float*>(slot_table + kMaxGrid);      // [5 warps][16 rows]
+    float* mean = ssw + 5 * kMaxM;                                      // [16] LayerNorm row means
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool split = NORM && p.M <= 8;   // X operand as hi/lo row pairs (see the prologue)
+    constexpr bool LN = (NORM == 2);
+    // X operand as hi/lo row pairs (see the prologue); LayerNorm keeps row 7 (split) or 15 for beta
+    const bool split = NORM && p.M <= (LN ? 7 : 8);
+    const int beta_row = split ? 7 : 15;
     const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
     const int it_end = range_begin(blockIdx.x + 1, p.base, p.rem);
 
@@ -136,8 +143,39 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
         const int idx = threadIdx.x - 32;  // 0..159
         const int chunks = p.K >> 3;
         float ss[kMaxM];
+        float mu[kMaxM];
 #pragma unroll
-        for (int r = 0; r < kMaxM; ++r) ss[r] = 0.f;
+        for (int r = 0; r < kMaxM; ++r) { ss[r] = 0.f; mu[r] = 0.f; }
+        if (LN) {
+            // row means first (a pass of its own: the deviations x - mean are what gets squared and multiplied)
+            for (int c = idx; c < chunks; c += 160) {
+#pragma unroll
+                for (int r = 0; r < kMaxM; ++r) {
+                    if (r < p.M) {
+                        const uint4 xv = __ldg(reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(r) * p.K) + c);
+                        const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) mu[r] += __uint_as_float(xs[j] << 16) + __uint_as_float(xs[j] & 0xFFFF0000u);
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < kMaxM; ++r) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mu[r] += __shfl_xor_sync(0xffffffffu, mu[r], o);
+                if (lane == 0) ssw[(warp - 1) * kMaxM + r] = mu[r];
+            }
+            asm volatile("bar.sync 2, 160;" ::: "memory");
+            if (idx < kMaxM) {
+                float tot = 0.f;
+#pragma unroll
+                for (int w = 0; w < 5; ++w) tot += ssw[w * kMaxM + idx];
+                mean[idx] = tot / static_cast<float>(p.K);
+            }
+            asm volatile("bar.sync 2, 160;" ::: "memory");
+#pragma unroll
+            for (int r = 0; r < kMaxM; ++r) mu[r] = mean[r];
+        }
         for (int c = idx; c < chunks; c += 160) {
             const uint4 gv = __ldg(reinterpret_cast<const uint4*>(p.gamma) + c);
             uint4 xv[kMaxM];
@@ -158,7 +196,8 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                     uint32_t hi4[4], lo4[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
+                        float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
+                        if (LN && r < p.M) { x0 -= mu[r]; x1 -= mu[r]; }
                         const float g0 = __uint_as_float(gs[j] << 16), g1 = __uint_as_float(gs[j] & 0xFFFF0000u);
                         ss[r] += x0 * x0 + x1 * x1;
                         const float v0 = x0 * g0, v1 = x1 * g1;
@@ -178,7 +217,8 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                     uint32_t outv[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
+                        float x0 = __uint_as_float(xs[j] << 16), x1 = __uint_as_float(xs[j] & 0xFFFF0000u);
+                        if (LN && r < p.M) { x0 -= mu[r]; x1 -= mu[r]; }
                         const float g0 = __uint_as_float(gs[j] << 16), g1 = __uint_as_float(gs[j] & 0xFFFF0000u);
                         ss[r] += x0 * x0 + x1 * x1;
                         outv[j] = pack_bf16x2(x0 * g0, x1 * g1);
@@ -186,6 +226,12 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                     *reinterpret_cast<uint4*>(xg + kb * kXBytes + r * 128 + ((cc ^ (r & 7)) << 4)) =
                         make_uint4(outv[0], outv[1], outv[2], outv[3]);
                 }
+            }
+            if (LN) {   // the spare row carries beta (exact in bf16); its partner lo row, if any, stays zero
+                const uint4 bv = __ldg(reinterpret_cast<const uint4*>(p.beta) + c);
+                *reinterpret_cast<uint4*>(xg + kb * kXBytes + beta_row * 128 + ((cc ^ (beta_row & 7)) << 4)) = bv;
+                if (split)
+                    *reinterpret_cast<uint4*>(xg + kb * kXBytes + 15 * 128 + ((cc ^ 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
             }
         }
         // per-row sum of squares: warp shuffle tree, then the five warp partials in warp order (deterministic)
@@ -317,6 +363,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                         float y;
                         if (NW == 2) y = silu(a0 * r) * (a1 * r);
                         else y = a0 * r;
+                        if (LN) y += __uint_as_float(split ? v[0][7] : v[0][15]);   // beta @ W, from the spare operand row
                         p.Y[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
                     }
                 }
@@ -356,18 +403,19 @@ inline bool make_plan(int NW, bool norm, int K, int N, Plan* pl) {
     return stages >= 2;
 }
 
-template <int NW, bool NORM>
-ef_status launch(const void* X, const void* gamma, const void* W0, const void* W1, void* Y, int M, int K, int N, float eps,
-                 void* ws, size_t ws_bytes, void* stream) {
-    if (!X || !W0 || !Y || (NW == 2 && !W1) || (NORM && !gamma)) return EF_ERR_NULL;
+template <int NW, int NORM>
+ef_status launch(const void* X, const void* gamma, const void* beta, const void* W0, const void* W1, void* Y, int M, int K,
+                 int N, float eps, void* ws, size_t ws_bytes, void* stream) {
+    if (!X || !W0 || !Y || (NW == 2 && !W1) || (NORM && !gamma) || (NORM == 2 && !beta)) return EF_ERR_NULL;
     if (M <= 0 || K <= 0 || N <= 0) return EF_ERR_SHAPE;
     if (M > kMaxM || K % kBK != 0 || N % 8 != 0) return EF_ERR_UNSUPPORTED;
+    if (NORM == 2 && M > kMaxM - 1) return EF_ERR_UNSUPPORTED;   // LayerNorm keeps one operand row for beta
     Plan pl;
-    if (!make_plan(NW, NORM, K, N, &pl)) return EF_ERR_UNSUPPORTED;  // NORM: X operand of the whole K must fit in shared memory
+    if (!make_plan(NW, NORM != 0, K, N, &pl)) return EF_ERR_UNSUPPORTED;  // NORM: X operand of the whole K must fit in shared memory
     if (static_cast<long long>(pl.n_tiles) * pl.k_blocks >= (1LL << 30)) return EF_ERR_UNSUPPORTED;
     if (kHeaderBytes + pl.counters_bytes > 65536) return EF_ERR_UNSUPPORTED;  // counters must lie in the init window
     if (!aligned(X, 16) || !aligned(W0, 16) || !aligned(Y, 16) || (NW == 2 && !aligned(W1, 16)) ||
-        (NORM && !aligned(gamma, 16)))
+        (NORM && !aligned(gamma, 16)) || (NORM == 2 && !aligned(beta, 16)))
         return EF_ERR_ALIGN;
     if (!ws || ws_bytes < pl.total) return EF_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EF_ERR_ALIGN;
@@ -395,6 +443,7 @@ ef_status launch(const void* X, const void* gamma, const void* W0, const void* W
     Params p;
     p.X = static_cast<const __nv_bfloat16*>(X);
     p.gamma = static_cast<const __nv_bfloat16*>(gamma);
+    p.beta = static_cast<const __nv_bfloat16*>(beta);
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.M = M; p.K = K; p.N = N;
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
@@ -434,7 +483,7 @@ size_t ef_rmsnorm_matmul_workspace_bytes(int M, int K, int N) {
 }
 ef_status ef_rmsnorm_matmul(const void* X, const void* gamma, const void* W, void* Y, int M, int K, int N, float eps,
                             void* ws, size_t ws_bytes, void* stream) {
-    return ef::skinny::launch<1, true>(X, gamma, W, nullptr, Y, M, K, N, eps, ws, ws_bytes, stream);
+    return ef::skinny::launch<1, 1>(X, gamma, nullptr, W, nullptr, Y, M, K, N, eps, ws, ws_bytes, stream);
 }
 
 size_t ef_rmsnorm_gated_mlp_workspace_bytes(int M, int K, int N) {
@@ -444,7 +493,17 @@ size_t ef_rmsnorm_gated_mlp_workspace_bytes(int M, int K, int N) {
 }
 ef_status ef_rmsnorm_gated_mlp(const void* X, const void* gamma, const void* Wgate, const void* Wup, void* Y, int M, int K,
                                int N, float eps, void* ws, size_t ws_bytes, void* stream) {
-    return ef::skinny::launch<2, true>(X, gamma, Wgate, Wup, Y, M, K, N, eps, ws, ws_bytes, stream);
+    return ef::skinny::launch<2, 1>(X, gamma, nullptr, Wgate, Wup, Y, M, K, N, eps, ws, ws_bytes, stream);
+}
+
+size_t ef_layernorm_matmul_workspace_bytes(int M, int K, int N) {
+    ef::skinny::Plan pl;
+    if (M <= 0 || K <= 0 || N <= 0 || K % ef::skinny::kBK != 0 || !ef::skinny::make_plan(1, true, K, N, &pl)) return 0;
+    return pl.total;
+}
+ef_status ef_layernorm_matmul(const void* X, const void* gamma, const void* beta, const void* W, void* Y, int M, int K,
+                              int N, float eps, void* ws, size_t ws_bytes, void* stream) {
+    return ef::skinny::launch<1, 2>(X, gamma, beta, W, nullptr, Y, M, K, N, eps, ws, ws_bytes, stream);
 }
 
 size_t ef_gated_mlp_workspace_bytes(int M, int K, int N) {
@@ -454,7 +513,7 @@ size_t ef_gated_mlp_workspace_bytes(int M, int K, int N) {
 }
 ef_status ef_gated_mlp(const void* X, const void* Wgate, const void* Wup, void* Y, int M, int K, int N, void* ws,
                        size_t ws_bytes, void* stream) {
-    return ef::skinny::launch<2, false>(X, nullptr, Wgate, Wup, Y, M, K, N, 0.f, ws, ws_bytes, stream);
+    return ef::skinny::launch<2, 0>(X, nullptr, nullptr, Wgate, Wup, Y, M, K, N, 0.f, ws, ws_bytes, stream);
 }
 
 }  // extern "C"

@@ -100,6 +100,37 @@ def test_rmsnorm_factor_motion_table1():
 # ----------------------------------------------------------------------------
 # Program 2: gated MLP
 # ----------------------------------------------------------------------------
+def test_layernorm_matmul_pins():
+    """LayerNorm+GEMM oracle: library special case (numpy mean/var + matmul), hand example, invariants
+    (shift and positive-scale invariance at eps=0, beta enters as beta@W, constant rows give beta@W), and the
+    fused form the kernel uses: r * ((x - mu) * gamma) @ W + beta @ W."""
+    M, K, N = 4, 12, 5
+    X = RNG.standard_normal((M, K)) + 0.7; g = 1 + 0.1 * RNG.standard_normal(K); b = 0.2 * RNG.standard_normal(K)
+    W = RNG.standard_normal((K, N)); eps = 1e-5
+    y = oracle.layernorm_matmul(X, g, b, W, eps)
+    mu = X.mean(1, keepdims=True); var = X.var(1, keepdims=True)        # numpy: biased variance
+    ref = ((X - mu) / np.sqrt(var + eps) * g + b) @ W
+    np.testing.assert_allclose(y, ref, **TOL)
+    # hand example: x = [1, 3] -> mu = 2, var = 1, eps = 0: xn = [-1, 1]; gamma = [2, 3], beta = [10, 20], W = I
+    yh = oracle.layernorm_matmul(np.array([[1.0, 3.0]]), np.array([2.0, 3.0]), np.array([10.0, 20.0]), np.eye(2), 0.0)
+    np.testing.assert_allclose(yh, [[8.0, 23.0]], **TOL)
+    # eps = 0: adding a constant to a row, or scaling it by t > 0, changes nothing
+    y0 = oracle.layernorm_matmul(X, g, b, W, 0.0)
+    np.testing.assert_allclose(oracle.layernorm_matmul(X + 5.0, g, b, W, 0.0), y0, rtol=1e-9, atol=1e-9)
+    np.testing.assert_allclose(oracle.layernorm_matmul(3.5 * X, g, b, W, 0.0), y0, rtol=1e-9, atol=1e-9)
+    # beta is additive through the projection; a constant row has no deviation, so its output is beta @ W
+    np.testing.assert_allclose(y - oracle.layernorm_matmul(X, g, 0 * b, W, eps), np.tile(b @ W, (M, 1)), **TOL)
+    np.testing.assert_allclose(oracle.layernorm_matmul(np.full((2, K), 4.0), g, b, W, eps), np.tile(b @ W, (2, 1)), **TOL)
+    # factor motion: the inverse standard deviation scales the finished projection; the mean does NOT move out
+    r = 1 / np.sqrt(var + eps)
+    np.testing.assert_allclose(r * (((X - mu) * g) @ W) + b @ W, y, **TOL)
+    assert not np.allclose(r * ((X * g) @ W) + b @ W, y, atol=1e-3)
+    # mean subtracted, unit variance: the normalised rows (gamma=1, beta=0, W=I) have mean 0 and mean square var/(var+eps)
+    z = oracle.layernorm_matmul(X, np.ones(K), np.zeros(K), np.eye(K), eps)
+    np.testing.assert_allclose(z.mean(1), 0, atol=1e-12)
+    np.testing.assert_allclose((z ** 2).mean(1), (var / (var + eps))[:, 0], **TOL)
+
+
 def test_silu_golden_values_through_one_hot_rows():
     g = load_golden("silu_constants.txt")
     # X one-hot picks row k of the weights: y_n = SiLU(Wg[k,n]) * Wu[k,n]

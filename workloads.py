@@ -22,7 +22,7 @@ import numpy as np
 
 PROGRAMS = ("rmsnorm_matmul", "gated_mlp", "gqa_decode", "qknorm_attn", "lora_linear")
 # programs beyond the five benchmark configurations (the "next" rows of the scope table)
-EXTRA_PROGRAMS = ("rmsnorm_gated_mlp", "gqa_decode_varlen")
+EXTRA_PROGRAMS = ("rmsnorm_gated_mlp", "gqa_decode_varlen", "layernorm_matmul")
 _PROGRAM_ID = {name: i for i, name in enumerate(PROGRAMS + EXTRA_PROGRAMS)}
 
 
@@ -107,6 +107,10 @@ SHAPES = {
         "full": dict(M=8, K=4096, N=11008, eps=1e-6),
         "small": dict(M=5, K=192, N=200, eps=1e-6),
     },
+    "layernorm_matmul": {  # LayerNorm+GEMM at batch 8, BERT-large hidden size into its 4x intermediate layer
+        "full": dict(M=8, K=1024, N=4096, eps=1e-5),
+        "small": dict(M=5, K=192, N=328, eps=1e-5),
+    },
     "gqa_decode": {
         "full": dict(B=8, Hq=32, Hkv=8, L=4096, D=128, scale=1.0 / np.sqrt(128.0)),
         "small": dict(B=2, Hq=8, Hkv=2, L=333, D=128, scale=1.0 / np.sqrt(128.0)),
@@ -153,6 +157,14 @@ def make_inputs(program: str, seed: int = 0, size: str = "full", **overrides):
             "gamma": g(1, (K,), 1.0, 0.1),
             "Wgate": g(2, (K, N), 0.0, 1.0 / np.sqrt(K)),
             "Wup": g(3, (K, N), 0.0, 1.0 / np.sqrt(K)),
+        }
+    elif program == "layernorm_matmul":
+        M, K, N = p["M"], p["K"], p["N"]
+        t = {
+            "X": g(0, (M, K), 0.3, 1.0),      # a non-zero mean: the subtraction must matter
+            "gamma": g(1, (K,), 1.0, 0.1),
+            "beta": g(2, (K,), 0.0, 0.1),
+            "W": g(3, (K, N), 0.0, 1.0 / np.sqrt(K)),
         }
     elif program == "gqa_decode":
         B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
@@ -208,6 +220,9 @@ def algorithmic_work(program: str, p: dict) -> dict:
     if program == "rmsnorm_matmul":
         M, K, N = p["M"], p["K"], p["N"]
         return dict(flops=2 * M * K * N, bytes=2 * (K * N + M * K + K + M * N))
+    if program == "layernorm_matmul":
+        M, K, N = p["M"], p["K"], p["N"]
+        return dict(flops=2 * M * K * N, bytes=2 * (K * N + M * K + 2 * K + M * N))
     if program == "gated_mlp":
         M, K, N = p["M"], p["K"], p["N"]
         return dict(flops=4 * M * K * N, bytes=2 * (2 * K * N + M * K + M * N))

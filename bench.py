@@ -177,7 +177,9 @@ def run_ours(args):
     calls_per_graph = 20
     # programs and shapes beyond the five configs of a step: measured the same way, outside the step
     extras = [(q, q, {}) for q in wl.EXTRA_PROGRAMS] + [("gqa_decode[B=1]", "gqa_decode", {"B": 1}),
-                                                        ("gqa_decode[B=16]", "gqa_decode", {"B": 16})]
+                                                        ("gqa_decode[B=16]", "gqa_decode", {"B": 16}),
+                                                        ("lora_linear[M=1]", "lora_linear", {"M": 1}),
+                                                        ("lora_linear[M=16]", "lora_linear", {"M": 16})]
     impl = {q: q for q in wl.PROGRAMS}   # key in `programs` -> entry point
     for key, prog, over in extras:
         pp, tt = wl.make_inputs(prog, seed=rank, size="full", **over)

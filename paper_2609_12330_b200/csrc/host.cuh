@@ -49,6 +49,17 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Skinny-M tail of the LoRA-fused linear (csrc/skinny.cu), used by ef_lora_linear for M <= 16.
+namespace skinny {
+constexpr int kLoraTailMaxM = 16;
+size_t lora_tail_counters_bytes(int N);
+size_t lora_tail_partials_bytes();
+ef_status launch_lora_head(const void* X, const void* A, void* T, int M, int K, float alpha, uint32_t* status,
+                           uint32_t* counters, float* partials, const DeviceInfo& di, cudaStream_t stream);
+ef_status launch_lora_tail(const void* X, const void* W, const void* T, const void* Bm, void* Y, int M, int K, int N,
+                           uint32_t* status, uint32_t* counters, float* partials, const DeviceInfo& di, cudaStream_t stream);
+}  // namespace skinny
+
 #define EF_CUDA_CHECK(expr)                                  \
     do {                                                     \
         cudaError_t _e = (expr);                             \

@@ -328,7 +328,7 @@ lora_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 
 struct Plan {
     int tiles_m, tiles_n, m_pad, k_blocks, splits;
-    size_t t_off, part_off, total;
+    size_t t_off, part_off, tail_counters_off, tail_part_off, total;
 };
 inline Plan make_plan(int M, int K, int N, int num_sms) {
     Plan pl;
@@ -342,9 +342,14 @@ inline Plan make_plan(int M, int K, int N, int num_sms) {
     const int min_s = (pl.k_blocks + kTStages - 1) / kTStages;  // each split fits the stage ring
     if (s < min_s) s = min_s;
     pl.splits = s;
-    pl.t_off = kHeaderBytes;
+    // M <= 16 takes the skinny-M second kernel: its per-n-tile arrival counters sit right behind the header (inside
+    // the window ef_workspace_init clears), its partial slots at the end
+    const bool skinny_tail = M <= skinny::kLoraTailMaxM;
+    pl.tail_counters_off = kHeaderBytes;
+    pl.t_off = kHeaderBytes + (skinny_tail ? skinny::lora_tail_counters_bytes(N) : 0);
     pl.part_off = pl.t_off + ((static_cast<size_t>(pl.m_pad) * kRank * 2 + 255) & ~size_t(255));
-    pl.total = pl.part_off + static_cast<size_t>(pl.k_blocks) * pl.m_pad * kRank * 4;  // worst case: one split per k block
+    pl.tail_part_off = pl.part_off + static_cast<size_t>(pl.k_blocks) * pl.m_pad * kRank * 4;  // worst case: one split per k block
+    pl.total = pl.tail_part_off + (skinny_tail ? skinny::lora_tail_partials_bytes() : 0);
     return pl;
 }
 
@@ -414,6 +419,16 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
         attr_set[di.device] = true;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (M <= skinny::kLoraTailMaxM) {
+        // Few rows: both kernels are weight-streaming problems, not tensor-bound ones.  Same two-kernel form
+        // (T stored once, reused by every output tile), on the skinny-projection kernel.
+        if (pl.t_off > 65536) return EF_ERR_UNSUPPORTED;   // counters must lie in the init window
+        uint32_t* status = reinterpret_cast<uint32_t*>(w);
+        uint32_t* counters = reinterpret_cast<uint32_t*>(w + pl.tail_counters_off);
+        float* partials = reinterpret_cast<float*>(w + pl.tail_part_off);
+        if ((st = skinny::launch_lora_head(X, A, T, M, K, alpha, status, counters, partials, di, s)) != EF_OK) return st;
+        return skinny::launch_lora_tail(X, W, T, Bm, Y, M, K, N, status, counters, partials, di, s);
+    }
     {
         lora::TParams tp;
         tp.T = T;

@@ -42,7 +42,9 @@ struct Params {
     int n_tiles, k_blocks, total_units;
     int base, rem;       // block c owns base + (c < rem) consecutive (tile, k block) units
     int stages;
+    int lora;            // NW == 1, no norm: the last k block of every n tile is the rank-16 update (T, Bm tiles)
     float eps;
+    float out_scale;     // NW == 1, no norm: the result is multiplied by this before rounding (1 elsewhere)
     uint32_t* status;
     uint32_t* counters;  // one per n tile, zero between calls
     float* partials;     // [grid][2][NW][16][128]
@@ -65,7 +67,7 @@ __device__ __forceinline__ float silu(float z) { return z / (1.f + __expf(-z)); 
 template <int NW, int NORM>
 __global__ void __launch_bounds__(kThreads, 1)
 skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
-              const __grid_constant__ CUtensorMap tmX, const Params p) {
+              const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmT, const Params p) {
     constexpr int kStageBytes = NW * kWBytes + (NORM ? 0 : kXBytes);
     constexpr uint32_t kAccCols = NW * kMaxM;          // fp32 columns per accumulator buffer
     constexpr uint32_t kTmemCols = 64;                 // two buffers of <= 32 columns
@@ -116,6 +118,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
             tma_prefetch_desc(&tmW0);
             if (NW == 2) tma_prefetch_desc(&tmW1);
             if (!NORM) tma_prefetch_desc(&tmX);
+            if (NW == 1 && !NORM && p.lora) { tma_prefetch_desc(&tmW1); tma_prefetch_desc(&tmT); }
             int stage = 0; uint32_t phase = 0;
             int tile = it_begin / p.k_blocks, kb = it_begin - tile * p.k_blocks;
             for (int it = it_begin; it < it_end; ++it) {
@@ -123,13 +126,21 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                 uint8_t* st = stages + stage * kStageBytes;
                 mbar_expect_tx(&full[stage], kStageBytes);
                 const int n0 = tile * kBN, k0 = kb * kBK;
-                tma_load_2d(st, &tmW0, &full[stage], n0, k0);
-                tma_load_2d(st + kWAtomBytes, &tmW0, &full[stage], n0 + 64, k0);
-                if (NW == 2) {
-                    tma_load_2d(st + kWBytes, &tmW1, &full[stage], n0, k0);
-                    tma_load_2d(st + kWBytes + kWAtomBytes, &tmW1, &full[stage], n0 + 64, k0);
+                if (NW == 1 && !NORM && p.lora && kb == p.k_blocks - 1) {
+                    // the rank-16 update as one more k block: Bm rows 16..63 and T columns 16..63 lie outside
+                    // their tensors and are filled with zeros (the second weight map carries Bm here)
+                    tma_load_2d(st, &tmW1, &full[stage], n0, 0);
+                    tma_load_2d(st + kWAtomBytes, &tmW1, &full[stage], n0 + 64, 0);
+                    tma_load_2d(st + NW * kWBytes, &tmT, &full[stage], 0, 0);
+                } else {
+                    tma_load_2d(st, &tmW0, &full[stage], n0, k0);
+                    tma_load_2d(st + kWAtomBytes, &tmW0, &full[stage], n0 + 64, k0);
+                    if (NW == 2) {
+                        tma_load_2d(st + kWBytes, &tmW1, &full[stage], n0, k0);
+                        tma_load_2d(st + kWBytes + kWAtomBytes, &tmW1, &full[stage], n0 + 64, k0);
+                    }
+                    if (!NORM) tma_load_2d(st + NW * kWBytes, &tmX, &full[stage], k0, 0);
                 }
-                if (!NORM) tma_load_2d(st + NW * kWBytes, &tmX, &full[stage], k0, 0);
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 if (++kb == p.k_blocks) { kb = 0; ++tile; }
             }
@@ -354,7 +365,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                 for (int m = 0; m < kMaxM; ++m) {
                     if (m < p.M) {
                         // r_m is invariant along K: it scales each finished projection (factor motion)
-                        const float r = NORM ? rinv[m] : 1.f;
+                        const float r = NORM ? rinv[m] : (NW == 1 ? p.out_scale : 1.f);
                         float a0 = __uint_as_float(v[0][m]), a1 = __uint_as_float(v[NW - 1][m]);
                         if (split) {  // hi + lo halves of the X operand (m < 8 here)
                             a0 += __uint_as_float(v[0][(m + 8) & 15]);
@@ -446,6 +457,8 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
     p.beta = static_cast<const __nv_bfloat16*>(beta);
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.M = M; p.K = K; p.N = N;
+    p.lora = 0;
+    p.out_scale = 1.f;
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
     int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
     if (grid > kMaxGrid) grid = kMaxGrid;
@@ -467,8 +480,74 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
     p.partials = reinterpret_cast<float*>(w + kHeaderBytes + pl.counters_bytes);
     EF_CUDA_CHECK(launch_pdl(skinny_kernel<NW, NORM>, dim3(grid), dim3(kThreads), static_cast<size_t>(pl.smem_bytes),
-                             static_cast<cudaStream_t>(stream), tmW0, tmW1, tmX, p));
+                             static_cast<cudaStream_t>(stream), tmW0, tmW1, tmX, tmX, p));
     return EF_OK;
+}
+
+// The LoRA-fused linear for M <= 16 rows, both kernels on the weight-streaming kernel above:
+//   launch_lora_head: T = alpha * X @ A   (A is a [K,16] weight: one n tile; few blocks, so few partials to merge)
+//   launch_lora_tail: Y = [X | T] @ [W ; Bm], the rank-16 update as one extra k block.
+size_t lora_tail_counters_bytes(int N) { return 256 + ((static_cast<size_t>((N + kBN - 1) / kBN) * 4 + 255) & ~size_t(255)); }
+size_t lora_tail_partials_bytes() { return static_cast<size_t>(kMaxGrid) * 2 * kMaxM * kBN * 4; }
+static ef_status launch_plain(const void* X, const void* W, int w_rows, const void* T, const void* Bm, void* Y, int M, int K,
+                              int N, float out_scale, int grid_cap, uint32_t* status, uint32_t* counters, float* partials,
+                              const DeviceInfo& di, cudaStream_t stream) {
+    const bool lora = T != nullptr;
+    Plan pl;
+    if (M > kMaxM || K % kBK != 0 || N % 8 != 0) return EF_ERR_UNSUPPORTED;
+    if (!make_plan(1, false, K + (lora ? kBK : 0), N, &pl)) return EF_ERR_UNSUPPORTED;   // LoRA: one more k block than K / 64
+    if (static_cast<long long>(pl.n_tiles) * pl.k_blocks >= (1LL << 30)) return EF_ERR_UNSUPPORTED;
+    CUtensorMap tmW, tmB, tmX, tmT;
+    ef_status st;
+    const uint64_t wdims[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(w_rows)};
+    const uint64_t bdims[2] = {static_cast<uint64_t>(N), 16};
+    const uint64_t wstrides[1] = {static_cast<uint64_t>(N) * 2};
+    const uint32_t wbox[2] = {64, kBK};
+    if ((st = encode_tmap_bf16(&tmW, W, 2, wdims, wstrides, wbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    if ((st = encode_tmap_bf16(&tmB, lora ? Bm : W, 2, lora ? bdims : wdims, wstrides, wbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    const uint64_t xdims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
+    const uint64_t xstrides[1] = {static_cast<uint64_t>(K) * 2};
+    const uint64_t tdims[2] = {16, static_cast<uint64_t>(M)};
+    const uint64_t tstrides[1] = {16 * 2};
+    const uint32_t xbox[2] = {64, kMaxM};
+    if ((st = encode_tmap_bf16(&tmX, X, 2, xdims, xstrides, xbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    if ((st = encode_tmap_bf16(&tmT, lora ? T : X, 2, lora ? tdims : xdims, lora ? tstrides : xstrides, xbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    static bool attr_set[64] = {};
+    if (!attr_set[di.device]) {
+        EF_CUDA_CHECK(cudaFuncSetAttribute(skinny_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        attr_set[di.device] = true;
+    }
+    Params p;
+    p.X = static_cast<const __nv_bfloat16*>(X);
+    p.gamma = nullptr;
+    p.beta = nullptr;
+    p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.M = M; p.K = K; p.N = N;
+    p.lora = lora ? 1 : 0;
+    p.out_scale = out_scale;
+    p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
+    int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
+    if (grid > kMaxGrid) grid = kMaxGrid;
+    if (grid > grid_cap) grid = grid_cap;
+    p.base = pl.total_units / grid;
+    p.rem = pl.total_units % grid;
+    p.stages = pl.stages;
+    p.eps = 0.f;
+    p.status = status;
+    p.counters = counters;
+    p.partials = partials;
+    EF_CUDA_CHECK(launch_pdl(skinny_kernel<1, 0>, dim3(grid), dim3(kThreads), static_cast<size_t>(pl.smem_bytes), stream, tmW,
+                             tmB, tmX, tmT, p));
+    return EF_OK;
+}
+ef_status launch_lora_head(const void* X, const void* A, void* T, int M, int K, float alpha, uint32_t* status,
+                           uint32_t* counters, float* partials, const DeviceInfo& di, cudaStream_t stream) {
+    // one n tile of 16 live columns, K / 64 k blocks: 8 blocks keep the ordered merge short
+    return launch_plain(X, A, K, nullptr, nullptr, T, M, K, 16, alpha, 8, status, counters, partials, di, stream);
+}
+ef_status launch_lora_tail(const void* X, const void* W, const void* T, const void* Bm, void* Y, int M, int K, int N,
+                           uint32_t* status, uint32_t* counters, float* partials, const DeviceInfo& di, cudaStream_t stream) {
+    return launch_plain(X, W, K, T, Bm, Y, M, K, N, 1.f, kMaxGrid, status, counters + 64, partials, di, stream);
 }
 
 }  // namespace skinny

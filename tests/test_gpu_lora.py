@@ -35,3 +35,18 @@ def test_lora_many_tiles_persistent_loop():
 def test_lora_full_config():
     r = run_parity("lora_linear", 0, size="full")
     assert r["rel_l2"] < 5e-3
+
+
+@pytest.mark.parametrize("M", [1, 5, 8, 16, 17])
+def test_lora_few_rows_take_the_weight_streaming_tail(M):
+    # M <= 16: second kernel = skinny projection with the rank-16 update as one extra k block; 17: the tiled kernel
+    run_parity("lora_linear", seed=7, size="small", M=M, K=512, N=1000)
+
+
+def test_lora_decode_shape():
+    # the B=1 LoRA case of Section 7.2 at the benchmark's layer size
+    run_parity("lora_linear", seed=8, size="full", M=1)
+
+
+def test_lora_few_rows_adapter_dominates():
+    run_parity("lora_linear", seed=9, size="small", M=4, K=256, N=264, alpha=25.0)

@@ -148,6 +148,21 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V,
                          void* ws, size_t ws_bytes, void* stream);
 size_t ef_qknorm_attn_workspace_bytes(int B, int H, int S, int D);
 
+/* ---- Program 4b: the same attention with grouped KV heads, a sliding window and attention sinks ----
+ * Mask variants of Section 7.3 (sliding-window attention with sink tokens: the first `sinks` keys plus
+ * the last `window` keys of every query stay visible; key tiles in between are skipped, and the tiles of
+ * both visible ranges feed ONE rolling softmax reduction) and grouped-query heads in prefill
+ * (consecutive query heads share a K/V head).  With causal != 0:
+ *   key j is visible to query i  iff  j <= i and (window == 0 or j > i - window or j < sinks).
+ *   Q,O [B,Hq,S,D], K,V [B,Hkv,S,D], gamma_q/gamma_k [D].
+ * Supported: D == 128, Hq % Hkv == 0, scale > 0; window > 0 and sinks > 0 need causal != 0; sinks <= 128;
+ * sinks > 0 needs window > 0.  window >= S means no window.  ef_qknorm_attn is the case Hq == Hkv,
+ * window == 0, sinks == 0.  Workspace: ef_qknorm_attn_workspace_bytes(B, Hkv, S, D). */
+ef_status ef_qknorm_attn_ex(const void* Q, const void* K, const void* V,
+                            const void* gamma_q, const void* gamma_k, void* O,
+                            int B, int Hq, int Hkv, int S, int D, float eps, float scale, int causal,
+                            int window, int sinks, void* ws, size_t ws_bytes, void* stream);
+
 /* ---- Program 5: LoRA-fused linear ---------------------------------------------------------
  * Y = X @ W + alpha * (X @ A) @ Bm.
  * Definition: the LoRA workload (Section 7.1; Figure 2 factoring; Table 1 MatMul

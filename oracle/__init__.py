@@ -115,6 +115,19 @@ def qknorm_attn(Q, K, V, gamma_q, gamma_k, eps, scale, causal=1):
     return O
 
 
+def qknorm_attn_ex(Q, K, V, gamma_q, gamma_k, eps, scale, causal=1, window=0, sinks=0):
+    Q, pQ = _d(Q); K, pK = _d(K); V, pV = _d(V)
+    gamma_q, pgq = _d(gamma_q); gamma_k, pgk = _d(gamma_k)
+    B, Hq, S, D = Q.shape
+    Hkv = K.shape[1]
+    assert K.shape == (B, Hkv, S, D) and V.shape == K.shape and Hq % Hkv == 0
+    assert gamma_q.shape == (D,) and gamma_k.shape == (D,)
+    O = np.empty((B, Hq, S, D), dtype=np.float64)
+    _load().ef_oracle_qknorm_attn_ex(pQ, pK, pV, pgq, pgk, _d(O)[1], B, Hq, Hkv, S, D, ctypes.c_double(eps),
+                                     ctypes.c_double(scale), int(causal), int(window), int(sinks))
+    return O
+
+
 def lora_linear(X, W, A, Bm, alpha):
     X, pX = _d(X); W, pW = _d(W); A, pA = _d(A); Bm, pB = _d(Bm)
     M, K = X.shape; N = W.shape[1]; R = A.shape[1]
@@ -141,6 +154,9 @@ def run(program: str, params: dict, tensors_f64: dict) -> np.ndarray:
         return gqa_decode_varlen(t["Q"], t["K"], t["V"], t["seq_lens"], p["scale"])
     if program == "qknorm_attn":
         return qknorm_attn(t["Q"], t["K"], t["V"], t["gamma_q"], t["gamma_k"], p["eps"], p["scale"], p.get("causal", 1))
+    if program == "qknorm_attn_ex":
+        return qknorm_attn_ex(t["Q"], t["K"], t["V"], t["gamma_q"], t["gamma_k"], p["eps"], p["scale"], p.get("causal", 1),
+                              p.get("window", 0), p.get("sinks", 0))
     if program == "lora_linear":
         return lora_linear(t["X"], t["W"], t["A"], t["Bm"], p["alpha"])
     raise KeyError(program)

@@ -238,6 +238,61 @@ void ef_oracle_qknorm_attn(const double *Q, const double *K, const double *V,
     }
 }
 
+/* Program 4b (Program 4 with grouped KV heads, a sliding window and attention sinks; the mask variants of
+ * Section 7.3).  Query head h of batch b reads kv head h / (Hq/Hkv).  With causal != 0 key j is visible to query i
+ * iff j <= i and (window == 0 or j > i - window or j < sinks); with causal == 0 every key is visible (window and
+ * sinks are then ignored).  Softmax runs over the visible keys only.  Q,O [B,Hq,S,D], K,V [B,Hkv,S,D]. */
+void ef_oracle_qknorm_attn_ex(const double *Q, const double *K, const double *V,
+                              const double *gamma_q, const double *gamma_k, double *O,
+                              int B, int Hq, int Hkv, int S, int D, double eps, double scale, int causal,
+                              int window, int sinks) {
+    const int group = Hq / Hkv;
+    for (int bh = 0; bh < B * Hq; ++bh) {
+        const int b = bh / Hq, h = bh % Hq, g = h / group;
+        const size_t qoff = (size_t)bh * S * D, koff = ((size_t)b * Hkv + g) * (size_t)S * D;
+        double *kh = (double *)malloc((size_t)S * D * sizeof(double));
+#pragma omp parallel for schedule(static)
+        for (int j = 0; j < S; ++j) {
+            const double *k = K + koff + (size_t)j * D;
+            const double r = inv_rms(k, D, eps);
+            for (int d = 0; d < D; ++d) kh[(size_t)j * D + d] = k[d] * r * gamma_k[d];
+        }
+#pragma omp parallel for schedule(dynamic, 16)
+        for (int i = 0; i < S; ++i) {
+            double *s = (double *)malloc((size_t)S * sizeof(double));
+            double *qh = (double *)malloc((size_t)D * sizeof(double));
+            const double *q = Q + qoff + (size_t)i * D;
+            const double r = inv_rms(q, D, eps);
+            for (int d = 0; d < D; ++d) qh[d] = q[d] * r * gamma_q[d];
+            double mx = -INFINITY;
+            for (int j = 0; j < S; ++j) {
+                const int vis = !causal || (j <= i && (window == 0 || j > i - window || j < sinks));
+                if (!vis) { s[j] = -INFINITY; continue; }
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d) dot += qh[d] * kh[(size_t)j * D + d];
+                s[j] = dot * scale;
+                if (s[j] > mx) mx = s[j];
+            }
+            double norm = 0.0;
+            for (int j = 0; j < S; ++j) {
+                s[j] = (s[j] == -INFINITY) ? 0.0 : exp(s[j] - mx);
+                norm += s[j];
+            }
+            double *out = O + qoff + (size_t)i * D;
+            for (int d = 0; d < D; ++d) out[d] = 0.0;
+            for (int j = 0; j < S; ++j) {
+                if (s[j] == 0.0) continue;
+                const double pj = s[j] / norm;
+                const double *v = V + koff + (size_t)j * D;
+                for (int d = 0; d < D; ++d) out[d] += pj * v[d];
+            }
+            free(s);
+            free(qh);
+        }
+        free(kh);
+    }
+}
+
 /* Program 5 (LoRA-fused linear, Section 7.2): T = X@A;  Y = X@W + alpha * (T@B).
  * X [M,K], W [K,N], A [K,R], Bm [R,N] -> Y [M,N]; alpha multiplies directly. */
 void ef_oracle_lora_linear(const double *X, const double *W, const double *A, const double *Bm,

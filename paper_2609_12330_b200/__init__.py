@@ -22,7 +22,7 @@ EXPORTS = [
     "ef_layernorm_matmul", "ef_layernorm_matmul_workspace_bytes",
     "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_varlen", "ef_gqa_decode_static",
     "ef_gqa_decode_static_max_units",
-    "ef_qknorm_attn", "ef_qknorm_attn_workspace_bytes",
+    "ef_qknorm_attn", "ef_qknorm_attn_workspace_bytes", "ef_qknorm_attn_ex",
     "ef_lora_linear", "ef_lora_linear_workspace_bytes",
     "ef_workspace_init", "ef_check_status", "ef_status_string", "ef_last_cuda_error", "ef_version",
 ]
@@ -58,6 +58,7 @@ def lib():
         L.ef_gqa_decode_static_max_units.argtypes = []
         L.ef_qknorm_attn.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, f, f, i, vp, sz, vp]
         L.ef_qknorm_attn_workspace_bytes.argtypes = [i, i, i, i]
+        L.ef_qknorm_attn_ex.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, f, i, i, i, vp, sz, vp]
         L.ef_lora_linear.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, vp, sz, vp]
         L.ef_lora_linear_workspace_bytes.argtypes = [i, i, i, i]
         L.ef_workspace_init.argtypes = [vp, sz, vp]
@@ -246,6 +247,20 @@ def qknorm_attn(Q, K, V, gamma_q, gamma_k, eps, scale, causal, ws: Workspace, ou
     return O
 
 
+def qknorm_attn_ex(Q, K, V, gamma_q, gamma_k, eps, scale, causal, window, sinks, ws: Workspace, out=None):
+    """QK-normalised attention with grouped KV heads (K, V: [B,Hkv,S,D]), a sliding window and attention sinks."""
+    import torch
+
+    B, Hq, S, D = Q.shape
+    Hkv = K.shape[1]
+    O = out if out is not None else torch.empty((B, Hq, S, D), dtype=torch.bfloat16, device=Q.device)
+    wp, wb = _ws_args(ws, qknorm_attn_workspace_bytes(B, Hkv, S, D), "ef_qknorm_attn_ex")
+    _check(lib().ef_qknorm_attn_ex(_ptr(Q, "Q"), _ptr(K, "K"), _ptr(V, "V"), _ptr(gamma_q, "gamma_q"),
+                                   _ptr(gamma_k, "gamma_k"), _ptr(O, "O"), B, Hq, Hkv, S, D, float(eps), float(scale),
+                                   int(causal), int(window), int(sinks), wp, wb, _stream()), "ef_qknorm_attn_ex")
+    return O
+
+
 def lora_linear(X, W, A, Bm, alpha, ws: Workspace, out=None):
     import torch
 
@@ -272,6 +287,8 @@ def workspace_bytes(program: str, p: dict) -> int:
         return gqa_decode_workspace_bytes(p["B"], p["Hq"], p["Hkv"], p["L"], p["D"])
     if program == "qknorm_attn":
         return qknorm_attn_workspace_bytes(p["B"], p["H"], p["S"], p["D"])
+    if program == "qknorm_attn_ex":
+        return qknorm_attn_workspace_bytes(p["B"], p["Hkv"], p["S"], p["D"])
     if program == "lora_linear":
         return lora_linear_workspace_bytes(p["M"], p["K"], p["N"], p["R"])
     raise KeyError(program)
@@ -294,6 +311,9 @@ def run(program: str, p: dict, t: dict, ws: Workspace, out=None):
     if program == "qknorm_attn":
         return qknorm_attn(t["Q"], t["K"], t["V"], t["gamma_q"], t["gamma_k"], p["eps"], p["scale"],
                            p.get("causal", 1), ws, out)
+    if program == "qknorm_attn_ex":
+        return qknorm_attn_ex(t["Q"], t["K"], t["V"], t["gamma_q"], t["gamma_k"], p["eps"], p["scale"], p.get("causal", 1),
+                              p.get("window", 0), p.get("sinks", 0), ws, out)
     if program == "lora_linear":
         return lora_linear(t["X"], t["W"], t["A"], t["Bm"], p["alpha"], ws, out)
     raise KeyError(program)

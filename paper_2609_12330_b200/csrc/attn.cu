@@ -60,6 +60,8 @@ struct Params {
     const __nv_bfloat16* gamma_k;
     __nv_bfloat16* O;     // [BH][S][128]
     int BH, S, nq, n_pairs, causal;
+    int Hq, Hkv;          // BH = B * Hq query heads; K and V have B * Hkv heads (consecutive query heads share one)
+    int window, sinks;    // causal only: key j is visible to query i iff j <= i and (j > i - window or j < sinks); 0 = no window
     float eps, scale_log2;
     int total_items;
     int o_vec8;           // O is 32-byte aligned: the epilogue may use 256-bit stores
@@ -166,27 +168,71 @@ __global__ void __launch_bounds__(256) key_normalize_kernel(const __nv_bfloat16*
 // ---------------------------------------------------------------------------------------------
 // Work item = (batch*head, pair of Q tiles); item index order is heaviest pair first, so greedy
 // pulling is longest-processing-time-first scheduling.
+// A pair visits a LIST of key tiles, shared by its two Q tiles: the tiles of the (causal, windowed) range of either
+// tile, preceded by key tile 0 when attention sinks are in use and the window has moved past it.  Entry a of the
+// list is key tile kt(a); Q tile t takes part in entry a iff part(t, a).
 struct Item {
-    int bh, qt0, n_kv, nkv0, nkv1;
+    int bh, qt0;
+    int n_kv;        // entries of the list
+    int lo;          // first key tile of the window range
+    int sink;        // 1: entry 0 is key tile 0, visited for the sink keys only
+    int wf0, wl0, wf1, wl1;   // first and last entry of tile t's window range (wl < wf: the tile is absent)
+    __device__ __forceinline__ int wf(int t) const { return t ? wf1 : wf0; }
+    __device__ __forceinline__ int wl(int t) const { return t ? wl1 : wl0; }
+    __device__ __forceinline__ int kt(int a) const { return sink ? (a == 0 ? 0 : lo + a - 1) : lo + a; }
+    __device__ __forceinline__ bool present(int t) const { return wl(t) >= wf(t); }
+    __device__ __forceinline__ bool part(int t, int a) const { return (sink && a == 0 && present(t)) || (a >= wf(t) && a <= wl(t)); }
+    __device__ __forceinline__ int first(int t) const { return (sink && present(t)) ? 0 : wf(t); }
+    __device__ __forceinline__ int last(int t) const { return wl(t); }
 };
-// geometry of the pair whose first Q tile is qt0 (no division: the consumers' per-item path)
+// geometry of the pair whose first Q tile is qt0 (no division: the consumers' per-item path).  WIN = false is the
+// kernel instance without a sliding window: the list is key tiles 0..hi, every field below folds to a constant
+// and part(t, a) is a single comparison again.
+template <bool WIN>
 __device__ __forceinline__ Item item_from(const Params& p, int bh, int qt0) {
     Item g;
     g.bh = bh;
     g.qt0 = qt0;
-    const int qt1 = qt0 + 1;
-    const bool has_q1 = qt1 < p.nq;
-    const int q_last = has_q1 ? qt1 : qt0;
-    g.n_kv = p.causal ? (q_last + 1) : p.nq;                       // key tiles the pair visits
-    g.nkv0 = p.causal ? (qt0 + 1) : p.nq;                          // ... and each of its two Q tiles
-    g.nkv1 = has_q1 ? (p.causal ? (qt1 + 1) : p.nq) : 0;
+    if constexpr (!WIN) {
+        const bool has_q1 = qt0 + 1 < p.nq;
+        const int hi0 = p.causal ? qt0 : p.nq - 1;
+        const int hi1 = has_q1 ? (p.causal ? qt0 + 1 : p.nq - 1) : -1;
+        g.lo = 0; g.sink = 0;
+        g.n_kv = max(hi0, hi1) + 1;
+        g.wf0 = 0; g.wl0 = hi0;
+        g.wf1 = 0; g.wl1 = hi1;
+        return g;
+    } else {
+    int lo_t[2], hi_t[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int qt = qt0 + t;
+        hi_t[t] = p.causal ? qt : p.nq - 1;
+        const int jmin = p.window > 0 ? max(0, qt * kT - p.window + 1) : 0;   // lowest key any row of the tile sees
+        lo_t[t] = jmin / kT;
+        if (qt >= p.nq) hi_t[t] = lo_t[t] - 1;                                 // absent tile
+    }
+    g.lo = lo_t[0];
+    g.sink = (p.sinks > 0 && g.lo > 0) ? 1 : 0;
+    const int hi = max(hi_t[0], hi_t[1]);
+    g.n_kv = hi - g.lo + 1 + g.sink;
+    g.wf0 = lo_t[0] - g.lo + g.sink; g.wl0 = hi_t[0] - g.lo + g.sink;
+    g.wf1 = lo_t[1] - g.lo + g.sink; g.wl1 = hi_t[1] - g.lo + g.sink;
+    // key tile 0 is inside the list but below a tile's window: it still holds that tile's sink keys
+    if (!g.sink && p.sinks > 0 && g.lo == 0) {
+        if (g.wl0 >= g.wf0) g.wf0 = 0;
+        if (g.wl1 >= g.wf1) g.wf1 = 0;
+    }
     return g;
+    }
 }
+template <bool WIN>
 __device__ __forceinline__ Item item_geom(const Params& p, int item) {
     const int pair = p.n_pairs - 1 - item / p.BH;
-    return item_from(p, item - (item / p.BH) * p.BH, 2 * pair);
+    return item_from<WIN>(p, item - (item / p.BH) * p.BH, 2 * pair);
 }
 
+template <bool WIN>
 __global__ void __launch_bounds__(kThreads, 1)
 qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const Params p) {
@@ -246,7 +292,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 const int slot = n_items & 1;
                 if (!mbar_wait(&item_empty[slot], ((n_items >> 1) & 1) ^ 1u, abort_flag, p.status, 1)) break;
                 const bool valid = item < static_cast<uint32_t>(p.total_items);
-                const Item g = item_geom(p, valid ? static_cast<int>(item) : 0);
+                const Item g = item_geom<WIN>(p, valid ? static_cast<int>(item) : 0);
                 item_ring[slot] = valid ? make_int2(g.bh, g.qt0) : make_int2(-1, 0);
                 mbar_arrive(&item_full[slot]);
                 if (!valid) break;
@@ -262,21 +308,23 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     return true;
                 };
                 if (!load_q(0)) break;
-                for (int j = 0; j < g.n_kv; ++j, ++kv_count) {
+                const int kvz = (p.Hq == p.Hkv) ? g.bh : (g.bh / p.Hq) * p.Hkv + (g.bh % p.Hq) / (p.Hq / p.Hkv);   // K/V head
+                for (int a = 0; a < g.n_kv; ++a, ++kv_count) {
+                    const int j = g.kt(a);   // key tile of list entry a
                     {
                         const uint32_t n = 2 * kv_count, sl = n % kKVSlots;
                         if (!mbar_wait(&kv_empty[sl], ((n / kKVSlots) & 1) ^ 1u, abort_flag, p.status, 3)) { ok = false; break; }
                         mbar_expect_tx(&kv_full[sl], kTileBytes);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmK, &kv_full[sl], 0, j * kT, g.bh);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmK, &kv_full[sl], 64, j * kT, g.bh);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmK, &kv_full[sl], 0, j * kT, kvz);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmK, &kv_full[sl], 64, j * kT, kvz);
                     }
-                    if (j == 0 && !load_q(1)) { ok = false; break; }
+                    if (a == 0 && !load_q(1)) { ok = false; break; }
                     {
                         const uint32_t n = 2 * kv_count + 1, sl = n % kKVSlots;
                         if (!mbar_wait(&kv_empty[sl], ((n / kKVSlots) & 1) ^ 1u, abort_flag, p.status, 3)) { ok = false; break; }
                         mbar_expect_tx(&kv_full[sl], kTileBytes);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmV, &kv_full[sl], 0, j * kT, g.bh);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmV, &kv_full[sl], 64, j * kT, g.bh);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmV, &kv_full[sl], 0, j * kT, kvz);
+                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmV, &kv_full[sl], 64, j * kT, kvz);
                     }
                 }
                 item = next;
@@ -324,17 +372,18 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 const int2 item = item_ring[slot];
                 mbar_arrive(&item_empty[slot]);
                 if (item.x < 0) break;
-                const Item g = item_from(p, item.x, item.y);
-                const int nkv[2] = {g.nkv0, g.nkv1};
-                // S_t(0): tile 0 starts as soon as ITS Q tile is rewritten and ITS old O has been read out
+                const Item g = item_from<WIN>(p, item.x, item.y);
+                // Entry a of the item's key list: tile t takes part iff g.part(t, a).  QK^T of entry a+1 is always
+                // issued during step a (right after the tile's PV of entry a, if it has one), so the K/V ring is
+                // released in list order whatever subset of entries a tile visits.
                 {
-                    const uint32_t n0 = 2 * kv_use, st0 = n0 % kKVSlots;   // K of the item's first key tile
+                    const uint32_t n0 = 2 * kv_use, st0 = n0 % kKVSlots;   // K of the item's first list entry
                     bool k_waited = false;
                     for (int t = 0; t < 2 && ok; ++t) {
                         ok = mbar_wait(&q_ready[t], n_items & 1, abort_flag, p.status, 4);
                         if (ok && n_items > 0) ok = mbar_wait(&o_free[t], (n_items - 1) & 1, abort_flag, p.status, 4);
                         if (!ok) break;
-                        if (nkv[t] > 0) {
+                        if (g.part(t, 0)) {
                             if (!k_waited) {
                                 if (!mbar_wait(&kv_full[st0], (n0 / kKVSlots) & 1, abort_flag, p.status, 5)) { ok = false; break; }
                                 k_waited = true;
@@ -343,7 +392,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                             issue_qk(t, st0);
                             umma_commit(&s_full[t]);
                         }
-                        if (nkv[t] <= 1) umma_commit(&q_empty[t]);   // that was tile t's only (or no) QK^T
+                        // tile t's last QK^T (or none at all): its Q tile may be overwritten
+                        if (!g.present(t) || g.last(t) == 0) umma_commit(&q_empty[t]);
                     }
                     if (!ok) break;
                     umma_commit(&kv_empty[st0]);
@@ -353,17 +403,18 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     const uint32_t st = nv % kKVSlots, stn = nk % kKVSlots;
                     bool v_waited = false, k_waited = false;
                     for (int t = 0; t < 2 && ok; ++t) {
-                        if (j >= nkv[t]) continue;
-                        if (!mbar_wait(&p_full[t], cp[t] & 1, abort_flag, p.status, 6)) { ok = false; break; }
-                        ++cp[t];
-                        if (!v_waited) {
-                            if (!mbar_wait(&kv_full[st], (nv / kKVSlots) & 1, abort_flag, p.status, 7)) { ok = false; break; }
-                            v_waited = true;
+                        if (g.part(t, j)) {
+                            if (!mbar_wait(&p_full[t], cp[t] & 1, abort_flag, p.status, 6)) { ok = false; break; }
+                            ++cp[t];
+                            if (!v_waited) {
+                                if (!mbar_wait(&kv_full[st], (nv / kKVSlots) & 1, abort_flag, p.status, 7)) { ok = false; break; }
+                                v_waited = true;
+                            }
+                            tc_fence_after();
+                            issue_pv(t, st, j > g.first(t) ? 1u : 0u);
+                            umma_commit(&o_done[t]);
                         }
-                        tc_fence_after();
-                        issue_pv(t, st, j > 0 ? 1u : 0u);
-                        umma_commit(&o_done[t]);
-                        if (j + 1 < nkv[t]) {
+                        if (j + 1 < g.n_kv && g.part(t, j + 1)) {
                             if (!k_waited) {
                                 if (!mbar_wait(&kv_full[stn], (nk / kKVSlots) & 1, abort_flag, p.status, 8)) { ok = false; break; }
                                 k_waited = true;
@@ -371,12 +422,12 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                             }
                             issue_qk(t, stn);
                             umma_commit(&s_full[t]);
-                            if (j + 2 == nkv[t]) umma_commit(&q_empty[t]);   // tile t's last QK^T: its Q tile is free
+                            if (j + 1 == g.last(t)) umma_commit(&q_empty[t]);   // tile t's last QK^T: its Q tile is free
                         }
                     }
                     if (!ok) break;
-                    umma_commit(&kv_empty[st]);                  // all PV of key tile j issued: V_j's slot is free
-                    if (k_waited) umma_commit(&kv_empty[stn]);   // all QK of key tile j+1 issued: K_j+1's slot is free
+                    umma_commit(&kv_empty[st]);                  // all PV of entry j issued: V_j's slot is free
+                    if (k_waited) umma_commit(&kv_empty[stn]);   // all QK of entry j+1 issued: K_j+1's slot is free
                 }
                 if (!ok) break;
                 kv_use += static_cast<uint32_t>(g.n_kv);
@@ -413,12 +464,13 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(&item_empty[slot]);
             if (item.x < 0) break;
-            const Item g = item_from(p, item.x, item.y);
-            const int my_nkv = (t == 0) ? g.nkv0 : g.nkv1;
+            const Item g = item_from<WIN>(p, item.x, item.y);
+            const bool present = g.present(t);
+            const int my_count = present ? g.wl(t) - g.wf(t) + 1 + g.sink : 0;   // list entries this tile takes part in
             const int qt = g.qt0 + t;
             const int row_g = qt * kT + r;             // query index within the sequence
             if (!warp_wait(&q_full[t], n_items & 1, abort_flag, p.status, 9)) break;
-            if (my_nkv > 0) {
+            if (present) {
                 // in-place rewrite of this thread's query row: qhat_d = fp16(q_d * rq_i); |q * rq| <= sqrt(128)
                 // whatever the scale of q, so fp16 is safe (the gammas ride on the keys)
                 uint8_t* qrow = smem + kOffQ + t * kTileBytes + r * 128;
@@ -449,7 +501,10 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(&q_ready[t]);   // every warp, every item (also when this tile has no work)
             float m_ref = fixed_ref ? bound : -INFINITY, l_sum = 0.f;
-            for (int j = 0; j < my_nkv && ok; ++j) {
+            int np = 0;   // entries processed so far
+            for (int a = g.first(t); a <= g.last(t) && ok; ++a) {
+                if (WIN && !g.part(t, a)) continue;
+                const int j = g.kt(a);   // key tile of this entry
                 if (!warp_wait(&s_full[t], cs & 1, abort_flag, p.status, 10)) { ok = false; break; }
                 ++cs;
                 tc_fence_after();
@@ -457,14 +512,34 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s[c]);
                 tmem_wait_ld();
+                // Masked tiles only: the diagonal tile, the ragged last key tile, and under a sliding window the
+                // tiles that reach below some row's window (the sink tile among them: only its sink keys count).
                 const bool diag = p.causal && (j == qt);
-                if (diag || (j * kT + kT > p.S)) {  // diagonal tile or ragged last key tile only
+                if constexpr (!WIN) {
+                    if (diag || (j * kT + kT > p.S)) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                        for (int c = 0; c < 4; ++c) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int col = c * 32 + i;
-                            if (!((!diag || col <= r) && (j * kT + col < p.S))) s[c][i] = 0xFF800000u;  // -inf
+                            for (int i = 0; i < 32; ++i) {
+                                const int col = c * 32 + i;
+                                if (!((!diag || col <= r) && (j * kT + col < p.S))) s[c][i] = 0xFF800000u;  // -inf
+                            }
+                        }
+                    }
+                } else {
+                    const bool below = j * kT <= qt * kT + kT - 1 - p.window;
+                    if (diag || below || (j * kT + kT > p.S)) {
+                        // column c of this tile is visible to this row iff c <= hi and (c >= lo or c < sk)
+                        const int hi = min(diag ? r : kT - 1, p.S - 1 - j * kT);
+                        const int lo = qt * kT + r - p.window + 1 - j * kT;
+                        const int sk = p.sinks - j * kT;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                const int col = c * 32 + i;
+                                if (!(col <= hi && (col >= lo || col < sk))) s[c][i] = 0xFF800000u;  // -inf
+                            }
                         }
                     }
                 }
@@ -488,7 +563,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     }
                 }
                 // p = exp2(acc * scale*log2e - m_ref): packed FMA, two exp2, packed row sum (4 independent accumulators)
-                const uint64_t nm2 = pack_f32x2(__float_as_uint(-m_ref), __float_as_uint(-m_ref));
+                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;   // a row may see nothing in its first tiles
+                const uint64_t nm2 = pack_f32x2(__float_as_uint(-m_use), __float_as_uint(-m_use));
                 uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
                 uint32_t pk[64];
 #pragma unroll
@@ -515,8 +591,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     tmem_st32(tS + 32, hi);
                 }
                 // rescale the accumulated value when some row of this warp moved its reference maximum
-                if (j > 0 && __any_sync(0xffffffffu, need)) {
-                    if (!warp_wait(&o_done[t], (co + j - 1) & 1, abort_flag, p.status, 12)) { ok = false; break; }
+                if (np > 0 && __any_sync(0xffffffffu, need)) {
+                    if (!warp_wait(&o_done[t], (co + np - 1) & 1, abort_flag, p.status, 12)) { ok = false; break; }
                     tc_fence_after();
 #pragma unroll 1
                     for (int c = 0; c < 4; ++c) {
@@ -532,11 +608,12 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&p_full[t]);
+                ++np;
             }
             if (!ok) break;
             // epilogue: read O out of TMEM (then the next item may overwrite it), scale by 1/l, store
-            if (my_nkv > 0) {
-                if (!warp_wait(&o_done[t], (co + my_nkv - 1) & 1, abort_flag, p.status, 13)) break;
+            if (my_count > 0) {
+                if (!warp_wait(&o_done[t], (co + my_count - 1) & 1, abort_flag, p.status, 13)) break;
                 tc_fence_after();
                 const float inv = 1.f / l_sum;
                 uint8_t* orow = reinterpret_cast<uint8_t*>(p.O + (static_cast<size_t>(g.bh) * p.S + row_g) * kD);
@@ -567,7 +644,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         }
                     }
                 }
-                co += static_cast<uint32_t>(my_nkv);
+                co += static_cast<uint32_t>(my_count);
             }
             tc_fence_before();
             __syncwarp();
@@ -593,21 +670,24 @@ size_t ef_qknorm_attn_workspace_bytes(int B, int H, int S, int D) {
     return ef::kHeaderBytes + static_cast<size_t>(B) * H * S * D * 2;   // header + Khat (normalised keys, bf16)
 }
 
-ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void* gamma_q, const void* gamma_k, void* O,
-                         int B, int H, int S, int D, float eps, float scale, int causal, void* ws, size_t ws_bytes,
-                         void* stream) {
+ef_status ef_qknorm_attn_ex(const void* Q, const void* K, const void* V, const void* gamma_q, const void* gamma_k, void* O,
+                            int B, int Hq, int Hkv, int S, int D, float eps, float scale, int causal, int window, int sinks,
+                            void* ws, size_t ws_bytes, void* stream) {
     using namespace ef;
     if (!Q || !K || !V || !gamma_q || !gamma_k || !O) return EF_ERR_NULL;
-    if (B <= 0 || H <= 0 || S <= 0 || D <= 0) return EF_ERR_SHAPE;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || S <= 0 || D <= 0 || Hq % Hkv != 0 || window < 0 || sinks < 0) return EF_ERR_SHAPE;
     if (D != attn::kD || !(scale > 0.f)) return EF_ERR_UNSUPPORTED;
-    const long long BH = static_cast<long long>(B) * H;
+    if ((window > 0 || sinks > 0) && !causal) return EF_ERR_UNSUPPORTED;   // the window is defined for causal attention
+    if (sinks > attn::kT || (sinks > 0 && window == 0)) return EF_ERR_UNSUPPORTED;   // sink keys lie in the first key tile
+    const long long BH = static_cast<long long>(B) * Hq;
+    const long long BHkv = static_cast<long long>(B) * Hkv;
     const int nq = (S + attn::kT - 1) / attn::kT;
     const int n_pairs = (nq + 1) / 2;
     if (BH * n_pairs > 0x7fffffffLL || BH > 0x3fffffff) return EF_ERR_UNSUPPORTED;
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(gamma_q, 2) ||
         !aligned(gamma_k, 2))
         return EF_ERR_ALIGN;
-    if (!ws || ws_bytes < ef_qknorm_attn_workspace_bytes(B, H, S, D)) return EF_ERR_WORKSPACE;
+    if (!ws || ws_bytes < ef_qknorm_attn_workspace_bytes(B, Hkv, S, D)) return EF_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EF_ERR_ALIGN;
     DeviceInfo di;
     if (!current_device_info(&di)) return EF_ERR_CUDA;
@@ -615,24 +695,27 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
 
     CUtensorMap tmQ, tmK, tmV;
     const uint64_t dims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(S), static_cast<uint64_t>(BH)};
+    const uint64_t kdims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(S), static_cast<uint64_t>(BHkv)};
     const uint64_t strides[2] = {static_cast<uint64_t>(D) * 2, static_cast<uint64_t>(S) * D * 2};
     const uint32_t box[3] = {64, attn::kT, 1};
     ef_status st;
     if ((st = encode_tmap_bf16(&tmQ, Q, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
     uint8_t* w = static_cast<uint8_t*>(ws);
     __nv_bfloat16* Khat = reinterpret_cast<__nv_bfloat16*>(w + kHeaderBytes);
-    if ((st = encode_tmap_bf16(&tmK, Khat, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
-    if ((st = encode_tmap_bf16(&tmV, V, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    if ((st = encode_tmap_bf16(&tmK, Khat, 3, kdims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+    if ((st = encode_tmap_bf16(&tmV, V, 3, kdims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
 
     static bool attr_set[64] = {};
     if (!attr_set[di.device]) {
-        EF_CUDA_CHECK(cudaFuncSetAttribute(attn::qknorm_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        EF_CUDA_CHECK(cudaFuncSetAttribute(attn::qknorm_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           attn::kSmemBytes));
+        EF_CUDA_CHECK(cudaFuncSetAttribute(attn::qknorm_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            attn::kSmemBytes));
         attr_set[di.device] = true;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     {
-        const long long rows = BH * S;
+        const long long rows = BHkv * S;
         const long long blocks = (rows + 16 * attn::kKeyRowsPerThread - 1) / (16 * attn::kKeyRowsPerThread);
         if (blocks > 0x7fffffffLL) return EF_ERR_UNSUPPORTED;
         EF_CUDA_CHECK(launch_pdl(attn::key_normalize_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s,
@@ -644,6 +727,9 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     p.gamma_k = static_cast<const __nv_bfloat16*>(gamma_k);
     p.O = static_cast<__nv_bfloat16*>(O);
     p.BH = static_cast<int>(BH); p.S = S; p.nq = nq; p.n_pairs = n_pairs; p.causal = causal ? 1 : 0;
+    p.Hq = Hq; p.Hkv = Hkv;
+    p.window = (window >= S) ? 0 : window;   // a window that covers every key is no window
+    p.sinks = p.window > 0 ? sinks : 0;
     p.eps = eps;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = reinterpret_cast<uint32_t*>(w);
@@ -651,8 +737,17 @@ ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void
     p.total_items = static_cast<int>(BH * n_pairs);
     p.o_vec8 = aligned(O, 32) ? 1 : 0;
     const unsigned grid = static_cast<unsigned>(p.total_items < di.num_sms ? p.total_items : di.num_sms);
-    EF_CUDA_CHECK(launch_pdl(attn::qknorm_attn_kernel, dim3(grid), dim3(attn::kThreads), attn::kSmemBytes, s, tmQ, tmK, tmV, p));
+    if (p.window > 0)
+        EF_CUDA_CHECK(launch_pdl(attn::qknorm_attn_kernel<true>, dim3(grid), dim3(attn::kThreads), attn::kSmemBytes, s, tmQ, tmK, tmV, p));
+    else
+        EF_CUDA_CHECK(launch_pdl(attn::qknorm_attn_kernel<false>, dim3(grid), dim3(attn::kThreads), attn::kSmemBytes, s, tmQ, tmK, tmV, p));
     return EF_OK;
+}
+
+ef_status ef_qknorm_attn(const void* Q, const void* K, const void* V, const void* gamma_q, const void* gamma_k, void* O,
+                         int B, int H, int S, int D, float eps, float scale, int causal, void* ws, size_t ws_bytes,
+                         void* stream) {
+    return ef_qknorm_attn_ex(Q, K, V, gamma_q, gamma_k, O, B, H, H, S, D, eps, scale, causal, 0, 0, ws, ws_bytes, stream);
 }
 
 }  // extern "C"

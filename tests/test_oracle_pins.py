@@ -468,6 +468,43 @@ def test_qknorm_rolling_with_causal_tile_skipping():
 # ----------------------------------------------------------------------------
 # Program 5: LoRA-fused linear
 # ----------------------------------------------------------------------------
+def test_qknorm_attn_ex_mask_variants():
+    """Window + sinks + grouped heads: equals a dense softmax under an explicitly built mask (library routines);
+    no window / MHA reduces to the plain program; a window of 1 returns v_i; sinks add exactly the first keys;
+    GQA equals MHA on repeat-interleaved K, V."""
+    B, Hq, Hkv, S, D = 2, 4, 2, 13, 6
+    Q = RNG.standard_normal((B, Hq, S, D)); K = RNG.standard_normal((B, Hkv, S, D)); V = RNG.standard_normal((B, Hkv, S, D))
+    gq = 1 + 0.1 * RNG.standard_normal(D); gk = 1 + 0.1 * RNG.standard_normal(D)
+    eps, scale = 1e-6, 0.6
+
+    def dense(window, sinks):
+        qh = Q / np.sqrt((Q ** 2).mean(-1, keepdims=True) + eps) * gq
+        kh = K / np.sqrt((K ** 2).mean(-1, keepdims=True) + eps) * gk
+        kx, vx = np.repeat(kh, Hq // Hkv, axis=1), np.repeat(V, Hq // Hkv, axis=1)
+        logits = np.einsum("bhid,bhjd->bhij", qh, kx) * scale
+        i, j = np.arange(S)[:, None], np.arange(S)[None, :]
+        vis = (j <= i) & ((window == 0) | (j > i - window) | (j < sinks))
+        logits = np.where(vis, logits, -np.inf)
+        return np.einsum("bhij,bhjd->bhid", softmax(logits, axis=-1), vx)
+
+    for window, sinks in [(0, 0), (5, 0), (5, 2), (1, 0), (1, 3), (4, 4), (13, 0), (100, 2)]:
+        o = oracle.qknorm_attn_ex(Q, K, V, gq, gk, eps, scale, 1, window, sinks)
+        np.testing.assert_allclose(o, dense(window, sinks), **TOL)
+    # window 1, no sinks: every query sees only itself
+    o1 = oracle.qknorm_attn_ex(Q, K, V, gq, gk, eps, scale, 1, 1, 0)
+    np.testing.assert_allclose(o1, np.repeat(V, Hq // Hkv, axis=1), **TOL)
+    # MHA, no window: the plain program (same routine family, independent code path in the oracle)
+    Kx, Vx = np.repeat(K, Hq // Hkv, axis=1), np.repeat(V, Hq // Hkv, axis=1)
+    np.testing.assert_allclose(oracle.qknorm_attn_ex(Q, Kx, Vx, gq, gk, eps, scale, 1, 0, 0),
+                               oracle.qknorm_attn(Q, Kx, Vx, gq, gk, eps, scale, 1), **TOL)
+    # grouped heads == MHA on expanded K, V, under a window as well
+    np.testing.assert_allclose(oracle.qknorm_attn_ex(Q, K, V, gq, gk, eps, scale, 1, 5, 2),
+                               oracle.qknorm_attn_ex(Q, Kx, Vx, gq, gk, eps, scale, 1, 5, 2), **TOL)
+    # non-causal ignores window and sinks
+    np.testing.assert_allclose(oracle.qknorm_attn_ex(Q, Kx, Vx, gq, gk, eps, scale, 0, 3, 1),
+                               oracle.qknorm_attn(Q, Kx, Vx, gq, gk, eps, scale, 0), **TOL)
+
+
 def test_lora_library_special_cases():
     M, K, N, R = 3, 7, 5, 2
     X = RNG.standard_normal((M, K)); W = RNG.standard_normal((K, N)); A = RNG.standard_normal((K, R)); B = RNG.standard_normal((R, N))

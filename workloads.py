@@ -22,7 +22,7 @@ import numpy as np
 
 PROGRAMS = ("rmsnorm_matmul", "gated_mlp", "gqa_decode", "qknorm_attn", "lora_linear")
 # programs beyond the five benchmark configurations (the "next" rows of the scope table)
-EXTRA_PROGRAMS = ("rmsnorm_gated_mlp", "gqa_decode_varlen", "layernorm_matmul")
+EXTRA_PROGRAMS = ("rmsnorm_gated_mlp", "gqa_decode_varlen", "layernorm_matmul", "qknorm_attn_ex")
 _PROGRAM_ID = {name: i for i, name in enumerate(PROGRAMS + EXTRA_PROGRAMS)}
 
 
@@ -123,6 +123,10 @@ SHAPES = {
         "full": dict(B=2, H=32, S=2048, D=128, eps=1e-6, scale=1.0 / np.sqrt(128.0), causal=1),
         "small": dict(B=1, H=2, S=300, D=128, eps=1e-6, scale=1.0 / np.sqrt(128.0), causal=1),
     },
+    "qknorm_attn_ex": {  # long-context prefill: grouped KV heads, sliding window with sink tokens (Section 7.3)
+        "full": dict(B=1, Hq=32, Hkv=8, S=8192, D=128, eps=1e-6, scale=1.0 / np.sqrt(128.0), causal=1, window=1024, sinks=4),
+        "small": dict(B=1, Hq=4, Hkv=2, S=700, D=128, eps=1e-6, scale=1.0 / np.sqrt(128.0), causal=1, window=200, sinks=4),
+    },
     "lora_linear": {
         "full": dict(M=2048, K=4096, N=4096, R=16, alpha=2.0),
         "small": dict(M=200, K=192, N=328, R=16, alpha=2.0),
@@ -202,6 +206,15 @@ def make_inputs(program: str, seed: int = 0, size: str = "full", **overrides):
             "gamma_q": g(3, (D,), 1.0, 0.1),
             "gamma_k": g(4, (D,), 1.0, 0.1),
         }
+    elif program == "qknorm_attn_ex":
+        B, Hq, Hkv, S, D = p["B"], p["Hq"], p["Hkv"], p["S"], p["D"]
+        t = {
+            "Q": g(0, (B, Hq, S, D), 0.0, 1.0),
+            "K": g(1, (B, Hkv, S, D), 0.0, 1.0),
+            "V": g(2, (B, Hkv, S, D), 0.0, 1.0),
+            "gamma_q": g(3, (D,), 1.0, 0.1),
+            "gamma_k": g(4, (D,), 1.0, 0.1),
+        }
     elif program == "lora_linear":
         M, K, N, R = p["M"], p["K"], p["N"], p["R"]
         t = {
@@ -240,6 +253,16 @@ def algorithmic_work(program: str, p: dict) -> dict:
         B, H, S, D = p["B"], p["H"], p["S"], p["D"]
         pairs = S * (S + 1) // 2 if p.get("causal", 1) else S * S
         return dict(flops=4 * B * H * D * pairs, bytes=2 * (4 * B * H * S * D + 2 * D))
+    if program == "qknorm_attn_ex":
+        B, Hq, Hkv, S, D = p["B"], p["Hq"], p["Hkv"], p["S"], p["D"]
+        w, sk = p.get("window", 0), p.get("sinks", 0)
+        if not p.get("causal", 1):
+            pairs = S * S
+        elif w <= 0 or w >= S:
+            pairs = S * (S + 1) // 2
+        else:   # row i sees min(i + 1, w) window keys plus the sink keys that lie below its window
+            pairs = sum(min(i + 1, w) + min(sk, max(0, i + 1 - w)) for i in range(S))
+        return dict(flops=4 * B * Hq * D * pairs, bytes=2 * (2 * B * Hq * S * D + 2 * B * Hkv * S * D + 2 * D))
     if program == "lora_linear":
         M, K, N, R = p["M"], p["K"], p["N"], p["R"]
         return dict(flops=2 * M * K * N + 2 * M * K * R + 2 * M * R * N,

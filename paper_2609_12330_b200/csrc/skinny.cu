@@ -58,6 +58,26 @@ __device__ __forceinline__ int owner_of(int x, int base, int rem) {
 __device__ __forceinline__ int slot_of(int c, int tile, int base, int rem, int k_blocks) {
     return 2 * c + ((range_begin(c, base, rem) / k_blocks) == tile ? 0 : 1);
 }
+// A block's range is a sequence of SEGMENTS, one per n tile it touches.  Only the first and the last can be partial
+// (shared with the neighbouring blocks).  Processing order: the partial LAST segment first, then the rest in
+// natural order -- both owners of a shared tile then reach it at the very start of the kernel, and the partial
+// exchange, the arrival counter and the merging block's epilogue overlap with the streaming of the whole tiles
+// instead of forming a serial tail after it.
+struct Seg {
+    int it0, it1;
+};
+__device__ __forceinline__ int seg_count(int it_begin, int it_end, int k_blocks) {
+    return it_end > it_begin ? (it_end - 1) / k_blocks - it_begin / k_blocks + 1 : 0;
+}
+__device__ __forceinline__ Seg seg_of(int s, int nseg, int it_begin, int it_end, int k_blocks) {
+    const bool rotate = nseg >= 2 && (it_end % k_blocks) != 0;
+    const int k = rotate ? (s == 0 ? nseg - 1 : s - 1) : s;   // natural index of the s-th processed segment
+    const int tile = it_begin / k_blocks + k;
+    Seg g;
+    g.it0 = max(it_begin, tile * k_blocks);
+    g.it1 = min(it_end, (tile + 1) * k_blocks);
+    return g;
+}
 __device__ __forceinline__ float silu(float z) { return z / (1.f + __expf(-z)); }
 
 // NW = number of weight matrices sharing the X operand (1: RMSNorm+matmul, 2: gated MLP)
@@ -96,6 +116,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
     const int beta_row = split ? 7 : 15;
     const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
     const int it_end = range_begin(blockIdx.x + 1, p.base, p.rem);
+    const int nseg = seg_count(it_begin, it_end, p.k_blocks);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -120,9 +141,13 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
             if (!NORM) tma_prefetch_desc(&tmX);
             if (NW == 1 && !NORM && p.lora) { tma_prefetch_desc(&tmW1); tma_prefetch_desc(&tmT); }
             int stage = 0; uint32_t phase = 0;
-            int tile = it_begin / p.k_blocks, kb = it_begin - tile * p.k_blocks;
-            for (int it = it_begin; it < it_end; ++it) {
-                if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) break;
+            bool okp = true;
+            for (int sg = 0; sg < nseg && okp; ++sg) {
+              const Seg seg = seg_of(sg, nseg, it_begin, it_end, p.k_blocks);
+              const int tile = seg.it0 / p.k_blocks;
+              for (int it = seg.it0; it < seg.it1; ++it) {
+                const int kb = it - tile * p.k_blocks;
+                if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) { okp = false; break; }
                 uint8_t* st = stages + stage * kStageBytes;
                 mbar_expect_tx(&full[stage], kStageBytes);
                 const int n0 = tile * kBN, k0 = kb * kBK;
@@ -142,7 +167,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                     if (!NORM) tma_load_2d(st + NW * kWBytes, &tmX, &full[stage], k0, 0);
                 }
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-                if (++kb == p.k_blocks) { kb = 0; ++tile; }
+              }
             }
         }
     } else if (NORM) {
@@ -268,12 +293,12 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
             constexpr uint32_t idesc = make_idesc_bf16(kBN, kMaxM, 1, 0);  // A MN-major, B K-major
             int stage = 0; uint32_t phase = 0;
             int iter = 0;
-            int it = it_begin;
             bool ok = true;
-            while (it < it_end && ok) {
+            for (int sg = 0; sg < nseg && ok; ++sg) {
+                const Seg seg = seg_of(sg, nseg, it_begin, it_end, p.k_blocks);
+                const int it = seg.it0, seg_end = seg.it1;
                 const int tile = it / p.k_blocks;
                 const int kb0 = it - tile * p.k_blocks;
-                const int seg_end = min(it_end, (tile + 1) * p.k_blocks);
                 const int acc = iter & 1;
                 if (!mbar_wait(&acc_empty[acc], ((iter >> 1) & 1) ^ 1u, abort_flag, p.status, 2)) break;
                 tc_fence_after();
@@ -296,7 +321,6 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (ok) umma_commit(&acc_full[acc]);
-                it = seg_end;
                 ++iter;
             }
         }
@@ -304,12 +328,12 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
         const int q = warp & 3;
         const int et = q * 32 + lane;  // 0..127: TMEM lane = weight column within the tile
         int iter = 0;
-        int it = it_begin;
-        while (it < it_end) {
+        for (int sg = 0; sg < nseg; ++sg) {
+            const Seg seg = seg_of(sg, nseg, it_begin, it_end, p.k_blocks);
+            const int it = seg.it0, seg_end = seg.it1;
             const int tile = it / p.k_blocks;
             const int kb0 = it - tile * p.k_blocks;
             const int tile_end = (tile + 1) * p.k_blocks;
-            const int seg_end = min(it_end, tile_end);
             const bool whole = (kb0 == 0) && (seg_end == tile_end);
             const int acc = iter & 1;
             if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[acc], (iter >> 1) & 1, abort_flag, p.status, 4))) break;
@@ -383,7 +407,6 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                 asm volatile("bar.sync 1, 128;" ::: "memory");  // slot table / is_last reuse
                 if (finish && warp == 2 && lane == 0) p.counters[tile] = 0u;
             }
-            it = seg_end;
             ++iter;
         }
     }

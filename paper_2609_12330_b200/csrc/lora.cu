@@ -28,14 +28,21 @@ constexpr int kRank = 16;
 // main kernel
 // --------------------------------------------------------------------------------------------
 constexpr int kBN = 256;
-constexpr int kStages = 4;
 constexpr int kABytes = kBM * kBK * 2;            // 16 KiB: [128 rows][64 k] K-major, 128B swizzle
 constexpr int kBAtomBytes = kBK * 128;            //  8 KiB: [64 k][64 n] MN-major, 128B swizzle
 constexpr int kBBytes = (kBN / 64) * kBAtomBytes; // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kThreads = 192;                     // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 256;
-constexpr uint32_t kTmemCols = 512;               // two 256-column fp32 accumulators
+constexpr uint32_t kTmemCols = 512;
+// MT = 128-row sub-tiles per block tile.  MT = 1: 128x256 tiles, 4 stages of 48 KiB, two 256-column accumulators
+// (the epilogue of one tile overlaps the mainloop of the next).  MT = 2: 256x256 tiles, 3 stages of 64 KiB, one
+// accumulator of 2 x 256 columns: a third less operand traffic from L2 per flop (the mainloop is bound by the
+// L2 -> shared-memory stream, not by the tensor pipe), no epilogue overlap.
+template <int MT> struct MainCfg {
+    static constexpr int kStages = MT == 1 ? 4 : 3;
+    static constexpr int kStageBytes = MT * kABytes + kBBytes;
+    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 256;
+    static constexpr int kAccBufs = MT == 1 ? 2 : 1;
+};
 
 struct MainParams {
     __nv_bfloat16* Y;
@@ -46,9 +53,11 @@ struct MainParams {
     uint32_t* status;
 };
 
+template <int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                  const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmB, const MainParams p) {
+    constexpr int kStages = MainCfg<MT>::kStages, kStageBytes = MainCfg<MT>::kStageBytes, kAccBufs = MainCfg<MT>::kAccBufs;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
@@ -82,19 +91,21 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.tiles_m) * kBM, n0 = (tile / p.tiles_m) * kBN;
+                const int m0 = (tile % p.tiles_m) * (MT * kBM), n0 = (tile / p.tiles_m) * kBN;
                 for (int kb = 0; kb < total_kb; ++kb) {
                     if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     uint8_t* sA = smem + stage * kStageBytes;
-                    uint8_t* sB = sA + kABytes;
+                    uint8_t* sB = sA + MT * kABytes;
                     mbar_expect_tx(&full[stage], kStageBytes);
                     if (kb < p.k_blocks) {
-                        tma_load_2d(sA, &tmX, &full[stage], kb * kBK, m0);
+#pragma unroll
+                        for (int h = 0; h < MT; ++h) tma_load_2d(sA + h * kABytes, &tmX, &full[stage], kb * kBK, m0 + h * kBM);
 #pragma unroll
                         for (int j = 0; j < kBN / 64; ++j)
                             tma_load_2d(sB + j * kBAtomBytes, &tmW, &full[stage], n0 + 64 * j, kb * kBK);
                     } else {  // rank-16 slab: columns >= 16 of T and rows >= 16 of Bm are out of bounds -> zero
-                        tma_load_2d(sA, &tmT, &full[stage], 0, m0);
+#pragma unroll
+                        for (int h = 0; h < MT; ++h) tma_load_2d(sA + h * kABytes, &tmT, &full[stage], 0, m0 + h * kBM);
 #pragma unroll
                         for (int j = 0; j < kBN / 64; ++j)
                             tma_load_2d(sB + j * kBAtomBytes, &tmB, &full[stage], n0 + 64 * j, 0);
@@ -110,8 +121,8 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             int iter = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++iter) {
-                const int acc = iter & 1;
-                const uint32_t acc_phase = (iter >> 1) & 1;
+                const int acc = kAccBufs == 2 ? (iter & 1) : 0;
+                const uint32_t acc_phase = kAccBufs == 2 ? ((iter >> 1) & 1) : (iter & 1);
                 if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, p.status, 2)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kBN;
@@ -119,13 +130,16 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                     if (!mbar_wait(&full[stage], phase, abort_flag, p.status, 3)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sA = smem_u32(smem + stage * kStageBytes);
-                    const uint64_t a_desc = make_smem_desc(sA, 16, 1024, kSwizzle128B);
-                    const uint64_t b_desc = make_smem_desc(sA + kABytes, kBAtomBytes, 1024, kSwizzle128B);
+                    const uint64_t b_desc = make_smem_desc(sA + MT * kABytes, kBAtomBytes, 1024, kSwizzle128B);
                     const int nk = (kb < p.k_blocks) ? kBK / 16 : kRank / 16;
-                    for (int kk = 0; kk < nk; ++kk) {
-                        // A advances 16 k = 32 B inside the swizzled row; B advances 16 k-rows = 2048 B
-                        umma_ss(d_tmem, a_desc + static_cast<uint64_t>(kk * 2), b_desc + static_cast<uint64_t>(kk * 128),
-                                idesc, (kb | kk) != 0 ? 1u : 0u);
+#pragma unroll
+                    for (int h = 0; h < MT; ++h) {
+                        const uint64_t a_desc = make_smem_desc(sA + h * kABytes, 16, 1024, kSwizzle128B);
+                        for (int kk = 0; kk < nk; ++kk) {
+                            // A advances 16 k = 32 B inside the swizzled row; B advances 16 k-rows = 2048 B
+                            umma_ss(d_tmem + h * kBN, a_desc + static_cast<uint64_t>(kk * 2), b_desc + static_cast<uint64_t>(kk * 128),
+                                    idesc, (kb | kk) != 0 ? 1u : 0u);
+                        }
                     }
                     umma_commit(&empty[stage]);
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -137,31 +151,34 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
         int iter = 0;
         for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++iter) {
-            const int acc = iter & 1;
-            const uint32_t acc_phase = (iter >> 1) & 1;
-            const int m0 = (tile % p.tiles_m) * kBM, n0 = (tile / p.tiles_m) * kBN;
+            const int acc = kAccBufs == 2 ? (iter & 1) : 0;
+            const uint32_t acc_phase = kAccBufs == 2 ? ((iter >> 1) & 1) : (iter & 1);
+            const int m0 = (tile % p.tiles_m) * (MT * kBM), n0 = (tile / p.tiles_m) * kBN;
             const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.status, 4));
             if (!ok) break;
             tc_fence_after();
-            const int row = m0 + q * 32 + lane;
-            const uint32_t taddr = tmem_base + acc * kBN + (static_cast<uint32_t>(q * 32) << 16);
-            __nv_bfloat16* yrow = p.Y + static_cast<size_t>(row) * p.N + n0;
 #pragma unroll 1
-            for (int c = 0; c < kBN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(taddr + c * 32, r);
-                tmem_wait_ld();
-                if (row < p.M) {
+            for (int h = 0; h < MT; ++h) {
+                const int row = m0 + h * kBM + q * 32 + lane;
+                const uint32_t taddr = tmem_base + (acc + h) * kBN + (static_cast<uint32_t>(q * 32) << 16);
+                __nv_bfloat16* yrow = p.Y + static_cast<size_t>(row) * p.N + n0;
+#pragma unroll 1
+                for (int c = 0; c < kBN / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + c * 32, r);
+                    tmem_wait_ld();
+                    if (row < p.M) {
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        const int col = n0 + c * 32 + v * 8;
-                        if (col + 8 <= p.N) {
-                            uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-                            o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-                            o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-                            o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-                            *reinterpret_cast<uint4*>(yrow + c * 32 + v * 8) = o;
+                        for (int v = 0; v < 4; ++v) {
+                            const int col = n0 + c * 32 + v * 8;
+                            if (col + 8 <= p.N) {
+                                uint4 o;
+                                o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                                o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                                o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                                o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                                *reinterpret_cast<uint4*>(yrow + c * 32 + v * 8) = o;
+                            }
                         }
                     }
                 }
@@ -414,7 +431,8 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
     }
     static bool attr_set[64] = {};
     if (!attr_set[di.device]) {
-        EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::kSmemBytes));
+        EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_main_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::MainCfg<1>::kSmemBytes));
+        EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_main_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::MainCfg<2>::kSmemBytes));
         EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::kTSmemBytes));
         attr_set[di.device] = true;
     }
@@ -444,12 +462,21 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
         lora::MainParams mp;
         mp.Y = static_cast<__nv_bfloat16*>(Y);
         mp.M = M; mp.N = N;
-        mp.tiles_m = pl.tiles_m; mp.num_tiles = pl.tiles_m * pl.tiles_n;
+        // 256-row block tiles (a third less operand traffic per flop) unless that costs more waves of the grid
+        const int tiles1 = pl.tiles_m * pl.tiles_n, tm2 = (M + 2 * lora::kBM - 1) / (2 * lora::kBM), tiles2 = tm2 * pl.tiles_n;
+        const int waves1 = (tiles1 + di.num_sms - 1) / di.num_sms, waves2 = (tiles2 + di.num_sms - 1) / di.num_sms;
+        const int mt = (M > lora::kBM && 2 * waves2 <= waves1) ? 2 : 1;
+        mp.tiles_m = mt == 2 ? tm2 : pl.tiles_m;
+        mp.num_tiles = mp.tiles_m * pl.tiles_n;
         mp.k_blocks = pl.k_blocks; mp.has_lora = 1;
         mp.status = reinterpret_cast<uint32_t*>(w);
         const int grid = di.num_sms < mp.num_tiles ? di.num_sms : mp.num_tiles;
-        EF_CUDA_CHECK(launch_pdl(lora::lora_main_kernel, dim3(grid), dim3(lora::kThreads), lora::kSmemBytes, s, tmX, tmW, tmT,
-                                 tmB, mp));
+        if (mt == 2)
+            EF_CUDA_CHECK(launch_pdl(lora::lora_main_kernel<2>, dim3(grid), dim3(lora::kThreads), lora::MainCfg<2>::kSmemBytes, s,
+                                     tmX, tmW, tmT, tmB, mp));
+        else
+            EF_CUDA_CHECK(launch_pdl(lora::lora_main_kernel<1>, dim3(grid), dim3(lora::kThreads), lora::MainCfg<1>::kSmemBytes, s,
+                                     tmX, tmW, tmT, tmB, mp));
     }
     return EF_OK;
 }

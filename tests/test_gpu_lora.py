@@ -50,3 +50,10 @@ def test_lora_decode_shape():
 
 def test_lora_few_rows_adapter_dominates():
     run_parity("lora_linear", seed=9, size="small", M=4, K=256, N=264, alpha=25.0)
+
+
+@pytest.mark.parametrize("M,K,N", [(512, 256, 9728), (400, 192, 9736), (300, 128, 19464)])
+def test_lora_256_row_block_tiles(M, K, N):
+    # enough 128x256 tiles for two waves of the grid: the kernel instance with 256-row block tiles runs,
+    # with ragged rows in the last tile and a ragged last column tile
+    run_parity("lora_linear", seed=10, size="small", M=M, K=K, N=N, check_repeat=False)

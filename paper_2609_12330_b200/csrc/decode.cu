@@ -72,8 +72,11 @@ __device__ __forceinline__ int owner_of(int x, int base, int rem) {
     return x < big ? x / (base + 1) : rem + (x - big) / base;
 }
 // Where item x of the flattened chunk list lies.  Uniform lengths: every (batch, kv head) unit has n_chunks chunks.
-// Per-sequence lengths: batch entry b has nb_b = ceil(len_b / 128) chunks per unit, cum[b] = sum of nb over
-// earlier entries, and its Hkv units follow each other, so entry b owns items [Hkv*cum[b], Hkv*cum[b+1]).
+// Per-sequence lengths: a unit of batch entry b has nb_b = ceil(len_b / 128) chunks FOLLOWED BY ONE EMPTY ITEM (the
+// fixed per-unit cost -- query load, four-warp merge, output write -- is about one chunk's worth of time, and equal
+// item counts per block should mean equal time: a block that gets many one-chunk sequences gets half as many);
+// cum[b] = sum of (nb + 1) over earlier entries with keys, and the Hkv units of an entry follow each other, so entry b
+// owns items [Hkv*cum[b], Hkv*cum[b+1]).
 // Layout of `cum` (shared memory, per-sequence-length variant only): [0..B] prefix, [B+1] base, [B+2] rem,
 // [B+3 ..] clamped lengths.
 struct Where {
@@ -81,6 +84,7 @@ struct Where {
     int chunk;        // chunk of x within the unit
     int unit_begin;   // item index of the unit's first chunk
     int n_chunks;     // chunks of the unit
+    int n_items;      // items of the unit in the list (n_chunks, plus the empty item of the per-sequence-length variant)
     int len;          // keys of the unit
 };
 template <bool VARLEN>
@@ -91,6 +95,7 @@ __device__ __forceinline__ Where locate(int x, const Params& p, const int* cum) 
         w.unit_begin = w.unit * p.n_chunks;
         w.chunk = x - w.unit_begin;
         w.n_chunks = p.n_chunks;
+        w.n_items = p.n_chunks;
         w.len = p.L;
     } else {
         int lo = 0, hi = p.B;   // largest b with Hkv * cum[b] <= x (entries without keys own no items)
@@ -104,7 +109,8 @@ __device__ __forceinline__ Where locate(int x, const Params& p, const int* cum) 
         w.unit = lo * p.Hkv + kvh;
         w.chunk = rel - kvh * nb;
         w.unit_begin = x - w.chunk;
-        w.n_chunks = nb;
+        w.n_chunks = nb - 1;
+        w.n_items = nb;
         w.len = cum[p.B + 3 + lo];   // clamped length, cached by the prologue
     }
     return w;
@@ -163,7 +169,7 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     int len = p.seq_lens[b];
                     len = len < 0 ? 0 : (len > p.L ? p.L : len);
                     cum[p.B + 3 + b] = len;
-                    sum += (len + kChunk - 1) / kChunk;
+                    sum += len > 0 ? (len + kChunk - 1) / kChunk + 1 : 0;
                 }
             }
             int incl = sum;
@@ -177,7 +183,7 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 const int b = b0 + i;
                 if (b < p.B) {
                     cum[b] = run;
-                    run += (cum[p.B + 3 + b] + kChunk - 1) / kChunk;
+                    run += cum[p.B + 3 + b] > 0 ? (cum[p.B + 3 + b] + kChunk - 1) / kChunk + 1 : 0;
                 }
             }
             if (lane == 31) {
@@ -210,10 +216,21 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             tma_prefetch_desc(&tmV);
             int stage = 0;
             uint32_t phase = 0;
-            Where w = {0, 0, 0, 1, 0};
+            Where w = {0, 0, 0, 1, 1, 0};
             if (it_begin < it_end) w = locate<VARLEN>(it_begin, p, cum);
-            int unit = w.unit, chunk = w.chunk, unit_chunks = w.n_chunks;
+            int unit = w.unit, chunk = w.chunk, unit_chunks = w.n_chunks, unit_items = w.n_items;
             for (int it = it_begin; it < it_end; ++it) {
+                if (chunk >= unit_chunks) {   // the unit's empty item: nothing to load
+                    chunk = 0;
+                    ++unit;
+                    if (it + 1 < it_end) {
+                        const Where nx = locate<VARLEN>(it + 1, p, cum);
+                        unit = nx.unit;
+                        unit_chunks = nx.n_chunks;
+                        unit_items = nx.n_items;
+                    }
+                    continue;
+                }
                 if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) break;
                 uint8_t* st = stages + stage * kStageBytes;
                 const int key0 = chunk * kChunk;
@@ -224,14 +241,9 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 tma_load_3d(st + 2 * kHalfBytes, &tmV, &fullV[stage], 0, key0, unit);
                 tma_load_3d(st + 3 * kHalfBytes, &tmV, &fullV[stage], 64, key0, unit);
                 if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                if (++chunk == unit_chunks) {
+                if (++chunk == unit_items) {   // (uniform lengths: items == chunks; otherwise the empty item comes next)
                     chunk = 0;
                     ++unit;
-                    if (VARLEN && it + 1 < it_end) {   // the next unit may belong to another batch entry
-                        const Where nx = locate<VARLEN>(it + 1, p, cum);
-                        unit = nx.unit;
-                        unit_chunks = nx.n_chunks;
-                    }
                 }
             }
         }
@@ -247,10 +259,16 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             const Where w = locate<VARLEN>(it, p, cum);
             const int unit = w.unit;
             const int c0 = w.chunk;
-            const int unit_end = w.unit_begin + w.n_chunks;
+            const int unit_end = w.unit_begin + w.n_chunks;            // end of the unit's chunks in the list
+            const int items_end = w.unit_begin + w.n_items;            // ... and of its items
             const int len = w.len;   // keys of this unit
-            const int seg_end = unit_end < it_end ? unit_end : it_end;
+            const int seg_stop = items_end < it_end ? items_end : it_end;   // where this block leaves the unit
+            const int seg_end = unit_end < seg_stop ? unit_end : seg_stop;  // ... and its last chunk of the unit
             const int n_seg = seg_end - it;
+            if (n_seg <= 0) {   // only the unit's empty item falls into this block's range
+                it = seg_stop;
+                continue;
+            }
             const bool whole_unit = (c0 == 0) && (seg_end == unit_end);
             const int b = unit / p.Hkv, kvh = unit - b * p.Hkv;
             const int head0 = kvh * p.G;
@@ -433,7 +451,7 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 }
             }
             consumer_sync();  // merge buffer, slot table and is_last are reused by the next segment
-            it = seg_end;
+            it = seg_stop;
         }
     }
     // Teardown.  On an aborted run give copies that are still in flight time to land before the

@@ -118,6 +118,17 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O,
                         void* ws, size_t ws_bytes, void* stream);
 size_t ef_gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int L, int D);
 
+/* ---- Program 3c: decode attention over a sliding window with attention sinks -----------------
+ * The single query sits at position L - 1 and sees keys j >= L - window plus the first `sinks`
+ * keys (Section 7.3: sliding-window GQA; attention sinks -- only the chunks that cover the sink
+ * tokens and the most recent `window` tokens are visited, the masked middle is skipped, and both
+ * ranges contribute to one online reduction so they share one softmax normalisation).
+ *   Q [B,Hq,D], K,V [B,Hkv,L,D] -> O [B,Hq,D].  window == 0 or window >= L: no window (sinks
+ *   ignored) = ef_gqa_decode.  Supported shapes, workspace and errors as ef_gqa_decode. */
+ef_status ef_gqa_decode_window(const void* Q, const void* K, const void* V, void* O,
+                               int B, int Hq, int Hkv, int L, int D, float scale, int window, int sinks,
+                               void* ws, size_t ws_bytes, void* stream);
+
 /* ---- Program 3b: decode attention with per-sequence key lengths -----------------------------
  * The same rolling reducer over a batch whose sequences have different lengths (the serving
  * case behind the decode workloads of Section 7.1, batch sizes 1/8/16): batch entry b attends

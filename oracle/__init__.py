@@ -92,6 +92,15 @@ def gqa_decode(Q, K, V, scale):
     return O
 
 
+def gqa_decode_window(Q, K, V, scale, window, sinks):
+    Q, pQ = _d(Q); K, pK = _d(K); V, pV = _d(V)
+    B, Hq, D = Q.shape; _, Hkv, L, _ = K.shape
+    assert K.shape == (B, Hkv, L, D) and V.shape == K.shape and Hq % Hkv == 0
+    O = np.empty((B, Hq, D), dtype=np.float64)
+    _load().ef_oracle_gqa_decode_window(pQ, pK, pV, _d(O)[1], B, Hq, Hkv, L, D, ctypes.c_double(scale), int(window), int(sinks))
+    return O
+
+
 def gqa_decode_varlen(Q, K, V, seq_lens, scale):
     Q, pQ = _d(Q); K, pK = _d(K); V, pV = _d(V)
     B, Hq, D = Q.shape; _, Hkv, L, _ = K.shape
@@ -150,6 +159,8 @@ def run(program: str, params: dict, tensors_f64: dict) -> np.ndarray:
         return rmsnorm_gated_mlp(t["X"], t["gamma"], t["Wgate"], t["Wup"], p["eps"])
     if program == "gqa_decode":
         return gqa_decode(t["Q"], t["K"], t["V"], p["scale"])
+    if program == "gqa_decode_window":
+        return gqa_decode_window(t["Q"], t["K"], t["V"], p["scale"], p["window"], p["sinks"])
     if program == "gqa_decode_varlen":
         return gqa_decode_varlen(t["Q"], t["K"], t["V"], t["seq_lens"], p["scale"])
     if program == "qknorm_attn":

@@ -182,6 +182,32 @@ void ef_oracle_gqa_decode(const double *Q, const double *K, const double *V, dou
     }
 }
 
+/* Program 3c (decode attention over a sliding window with attention sinks, Section 7.3): the query is the last
+ * position L - 1; key j is visible iff window == 0 or window >= L or j >= L - window or j < sinks.  Softmax and the
+ * weighted sum run over the visible keys only (they are gathered first, then Program 3's row routine is applied). */
+void ef_oracle_gqa_decode_window(const double *Q, const double *K, const double *V, double *O,
+                                 int B, int Hq, int Hkv, int L, int D, double scale, int window, int sinks) {
+    const int group = Hq / Hkv;
+    const int windowed = window > 0 && window < L;
+#pragma omp parallel for schedule(static)
+    for (int bh = 0; bh < B * Hq; ++bh) {
+        const int b = bh / Hq, h = bh % Hq, g = h / group;
+        const size_t kv_off = ((size_t)b * Hkv + g) * (size_t)L * D;
+        double *kk = (double *)malloc((size_t)L * D * sizeof(double));
+        double *vv = (double *)malloc((size_t)L * D * sizeof(double));
+        double *s = (double *)malloc((size_t)L * sizeof(double));
+        int n = 0;
+        for (int j = 0; j < L; ++j) {
+            if (windowed && !(j >= L - window || j < sinks)) continue;
+            memcpy(kk + (size_t)n * D, K + kv_off + (size_t)j * D, (size_t)D * sizeof(double));
+            memcpy(vv + (size_t)n * D, V + kv_off + (size_t)j * D, (size_t)D * sizeof(double));
+            ++n;
+        }
+        attend_row(Q + (size_t)bh * D, kk, vv, (size_t)D, n, D, scale, s, O + (size_t)bh * D);
+        free(kk); free(vv); free(s);
+    }
+}
+
 /* Program 3b (decode attention, per-sequence key lengths): batch entry b attends keys [0, len_b) of its
  * K/V rows (len_b clamped to [0, L]); rows at and beyond len_b are padding and are never read.  An entry
  * with no keys has no softmax; its output is defined as zero.  Otherwise exactly Program 3 per entry. */

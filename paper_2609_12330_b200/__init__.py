@@ -20,7 +20,7 @@ EXPORTS = [
     "ef_gated_mlp", "ef_gated_mlp_workspace_bytes",
     "ef_rmsnorm_gated_mlp", "ef_rmsnorm_gated_mlp_workspace_bytes",
     "ef_layernorm_matmul", "ef_layernorm_matmul_workspace_bytes",
-    "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_varlen", "ef_gqa_decode_static",
+    "ef_gqa_decode", "ef_gqa_decode_workspace_bytes", "ef_gqa_decode_varlen", "ef_gqa_decode_window", "ef_gqa_decode_static",
     "ef_gqa_decode_static_max_units",
     "ef_qknorm_attn", "ef_qknorm_attn_workspace_bytes", "ef_qknorm_attn_ex",
     "ef_lora_linear", "ef_lora_linear_workspace_bytes",
@@ -53,6 +53,7 @@ def lib():
         L.ef_layernorm_matmul_workspace_bytes.argtypes = [i, i, i]
         L.ef_gqa_decode.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
         L.ef_gqa_decode_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.ef_gqa_decode_window.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp, sz, vp]
         L.ef_gqa_decode_varlen.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, vp, sz, vp]
         L.ef_gqa_decode_static.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, vp]
         L.ef_gqa_decode_static_max_units.argtypes = []
@@ -204,6 +205,19 @@ def gqa_decode(Q, K, V, scale, ws: Workspace, out=None):
     return O
 
 
+def gqa_decode_window(Q, K, V, scale, window, sinks, ws: Workspace, out=None):
+    """Decode attention over the last `window` keys plus the first `sinks` keys (the query is the last position)."""
+    import torch
+
+    B, Hq, D = Q.shape
+    _, Hkv, L, _ = K.shape
+    O = out if out is not None else torch.empty((B, Hq, D), dtype=torch.bfloat16, device=Q.device)
+    wp, wb = _ws_args(ws, gqa_decode_workspace_bytes(B, Hq, Hkv, L, D), "ef_gqa_decode_window")
+    _check(lib().ef_gqa_decode_window(_ptr(Q, "Q"), _ptr(K, "K"), _ptr(V, "V"), _ptr(O, "O"), B, Hq, Hkv, L, D,
+                                      float(scale), int(window), int(sinks), wp, wb, _stream()), "ef_gqa_decode_window")
+    return O
+
+
 def gqa_decode_varlen(Q, K, V, seq_lens, scale, ws: Workspace, out=None):
     """Decode attention where batch entry b attends keys [0, seq_lens[b]); seq_lens is a CUDA int32 tensor [B]."""
     import torch
@@ -283,7 +297,7 @@ def workspace_bytes(program: str, p: dict) -> int:
         return rmsnorm_gated_mlp_workspace_bytes(p["M"], p["K"], p["N"])
     if program == "layernorm_matmul":
         return layernorm_matmul_workspace_bytes(p["M"], p["K"], p["N"])
-    if program in ("gqa_decode", "gqa_decode_varlen"):
+    if program in ("gqa_decode", "gqa_decode_varlen", "gqa_decode_window"):
         return gqa_decode_workspace_bytes(p["B"], p["Hq"], p["Hkv"], p["L"], p["D"])
     if program == "qknorm_attn":
         return qknorm_attn_workspace_bytes(p["B"], p["H"], p["S"], p["D"])
@@ -306,6 +320,8 @@ def run(program: str, p: dict, t: dict, ws: Workspace, out=None):
         return layernorm_matmul(t["X"], t["gamma"], t["beta"], t["W"], p["eps"], ws, out)
     if program == "gqa_decode":
         return gqa_decode(t["Q"], t["K"], t["V"], p["scale"], ws, out)
+    if program == "gqa_decode_window":
+        return gqa_decode_window(t["Q"], t["K"], t["V"], p["scale"], p["window"], p["sinks"], ws, out)
     if program == "gqa_decode_varlen":
         return gqa_decode_varlen(t["Q"], t["K"], t["V"], t["seq_lens"], p["scale"], ws, out)
     if program == "qknorm_attn":

@@ -47,6 +47,9 @@ struct Params {
     const __nv_bfloat16* Q;
     __nv_bfloat16* O;
     int B, Hq, Hkv, L, G;
+    // sliding window + attention sinks (uniform-length kernel only; all zero = no window): the list of a unit is
+    // sink_chunks leading chunks followed by the chunks from win_chunk0 on; key j counts iff j >= win_start or j < sinks
+    int win_start, sinks, sink_chunks, win_chunk0;
     const int* seq_lens;   // per-sequence-length variant: keys [0, seq_lens[b]) of batch entry b are attended
     int n_chunks;      // chunks per (b, kv head) unit (uniform variant)
     int total_items;   // units * n_chunks  (< 2^30)
@@ -121,7 +124,7 @@ __device__ __forceinline__ int slot_of(int c, int unit, int base, int rem, const
     return 2 * c + (locate<VARLEN>(range_begin(c, base, rem), p, cum).unit == unit ? 0 : 1);
 }
 
-template <bool VARLEN>
+template <bool VARLEN, bool WIN>
 __global__ void __launch_bounds__(kThreads, 1)
 gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
     extern __shared__ uint8_t smem_raw[];
@@ -233,7 +236,7 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 }
                 if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) break;
                 uint8_t* st = stages + stage * kStageBytes;
-                const int key0 = chunk * kChunk;
+                const int key0 = (WIN ? (chunk < p.sink_chunks ? chunk : p.win_chunk0 + chunk - p.sink_chunks) : chunk) * kChunk;
                 mbar_expect_tx(&fullK[stage], 2 * kHalfBytes);
                 tma_load_3d(st, &tmK, &fullK[stage], 0, key0, unit);
                 tma_load_3d(st + kHalfBytes, &tmK, &fullK[stage], 64, key0, unit);
@@ -293,7 +296,8 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
 
             for (int ch = 0; ch < n_seg; ++ch) {
-                const int key_base = (c0 + ch) * kChunk + warp * kKeysPerWarp;
+                const int kc = WIN ? ((c0 + ch) < p.sink_chunks ? (c0 + ch) : p.win_chunk0 + (c0 + ch) - p.sink_chunks) : (c0 + ch);   // key chunk of this item
+                const int key_base = kc * kChunk + warp * kKeysPerWarp;
                 const uint32_t st = smem_u32(stages + stage * kStageBytes);
                 if (!warp_wait(&fullK[stage], phase, abort_flag, p.status, 2)) { ok = false; break; }
                 // ---- S = Q K^T for this warp's 32 keys: 4 n-tiles x 8 k-steps
@@ -318,8 +322,10 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll
                 for (int nt = 0; nt < 4; ++nt) {
                     const int key = key_base + nt * 8 + 2 * t4;
-                    s[nt][0] = (key < len) ? s[nt][0] * p.scale_log2 : -INFINITY;
-                    s[nt][1] = (key + 1 < len) ? s[nt][1] * p.scale_log2 : -INFINITY;
+                    const bool v0 = key < len && (!WIN || key >= p.win_start || key < p.sinks);
+                    const bool v1 = key + 1 < len && (!WIN || key + 1 >= p.win_start || key + 1 < p.sinks);
+                    s[nt][0] = v0 ? s[nt][0] * p.scale_log2 : -INFINITY;
+                    s[nt][1] = v1 ? s[nt][1] * p.scale_log2 : -INFINITY;
                     mx = fmaxf(mx, fmaxf(s[nt][0], s[nt][1]));
                 }
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -474,16 +480,26 @@ size_t ef_gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int L, int D) {
     return ef::kHeaderBytes + counters + static_cast<size_t>(ef::decode::kMaxGrid) * 2 * ef::decode::kSlotFloats * sizeof(float);
 }
 
-ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, int B, int Hq, int Hkv, int L, int D,
-                        float scale, void* ws, size_t ws_bytes, void* stream) {
+ef_status ef_gqa_decode_window(const void* Q, const void* K, const void* V, void* O, int B, int Hq, int Hkv, int L, int D,
+                               float scale, int window, int sinks, void* ws, size_t ws_bytes, void* stream) {
     using namespace ef;
     if (!Q || !K || !V || !O) return EF_ERR_NULL;
-    if (B <= 0 || Hq <= 0 || Hkv <= 0 || L <= 0 || D <= 0 || Hq % Hkv != 0) return EF_ERR_SHAPE;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || L <= 0 || D <= 0 || Hq % Hkv != 0 || window < 0 || sinks < 0) return EF_ERR_SHAPE;
     if (D != decode::kD || Hq / Hkv > decode::kMaxGroup) return EF_ERR_UNSUPPORTED;
     const size_t n_units = static_cast<size_t>(B) * Hkv;
     const size_t counters_bytes = (n_units * sizeof(uint32_t) + 255) & ~size_t(255);
     if (kHeaderBytes + counters_bytes > 65536) return EF_ERR_UNSUPPORTED;  // counters must lie in the init window
-    const long long n_chunks = (static_cast<long long>(L) + decode::kChunk - 1) / decode::kChunk;
+    // The single query sits at position L - 1: with a window it sees keys j >= L - window and the first `sinks` keys.
+    // Chunks between the sink chunks and the first window chunk are never loaded.
+    const long long all_chunks = (static_cast<long long>(L) + decode::kChunk - 1) / decode::kChunk;
+    int win_start = 0, sink_chunks = 0, win_chunk0 = 0;
+    if (window > 0 && window < L) {
+        win_start = L - window;
+        win_chunk0 = win_start / decode::kChunk;
+        sink_chunks = (sinks + decode::kChunk - 1) / decode::kChunk;
+        if (sink_chunks > win_chunk0) sink_chunks = win_chunk0;
+    }
+    const long long n_chunks = sink_chunks + (all_chunks - win_chunk0);
     if (n_chunks * static_cast<long long>(n_units) >= (1LL << 30)) return EF_ERR_UNSUPPORTED;
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16)) return EF_ERR_ALIGN;
     if (!ws || ws_bytes < ef_gqa_decode_workspace_bytes(B, Hq, Hkv, L, D)) return EF_ERR_WORKSPACE;
@@ -503,7 +519,9 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
 
     static bool attr_set[64] = {};
     if (!attr_set[di.device]) {
-        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           decode::kSmemBytes));
+        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            decode::kSmemBytes));
         attr_set[di.device] = true;
     }
@@ -512,6 +530,7 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
     p.O = static_cast<__nv_bfloat16*>(O);
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.L = L; p.G = Hq / Hkv;
     p.seq_lens = nullptr;
+    p.win_start = win_start; p.sinks = win_start > 0 ? sinks : 0; p.sink_chunks = sink_chunks; p.win_chunk0 = win_chunk0;
     p.n_chunks = static_cast<int>(n_chunks);
     p.total_items = static_cast<int>(n_chunks * static_cast<long long>(n_units));
     int grid = di.num_sms < p.total_items ? di.num_sms : p.total_items;
@@ -523,9 +542,18 @@ ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, in
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
     p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
-    EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<false>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
-                             static_cast<cudaStream_t>(stream), tmK, tmV, p));
+    if (win_start > 0)
+        EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<false, true>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
+                                 static_cast<cudaStream_t>(stream), tmK, tmV, p));
+    else
+        EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<false, false>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
+                                 static_cast<cudaStream_t>(stream), tmK, tmV, p));
     return EF_OK;
+}
+
+ef_status ef_gqa_decode(const void* Q, const void* K, const void* V, void* O, int B, int Hq, int Hkv, int L, int D,
+                        float scale, void* ws, size_t ws_bytes, void* stream) {
+    return ef_gqa_decode_window(Q, K, V, O, B, Hq, Hkv, L, D, scale, 0, 0, ws, ws_bytes, stream);
 }
 
 ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, const void* seq_lens, void* O, int B, int Hq,
@@ -557,7 +585,7 @@ ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, cons
 
     static bool attr_set[64] = {};
     if (!attr_set[di.device]) {
-        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        EF_CUDA_CHECK(cudaFuncSetAttribute(decode::gqa_decode_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            decode::kSmemBytes));
         attr_set[di.device] = true;
     }
@@ -566,6 +594,7 @@ ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, cons
     p.O = static_cast<__nv_bfloat16*>(O);
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.L = Lmax; p.G = Hq / Hkv;
     p.seq_lens = static_cast<const int*>(seq_lens);
+    p.win_start = 0; p.sinks = 0; p.sink_chunks = 0; p.win_chunk0 = 0;
     p.n_chunks = static_cast<int>(n_chunks);
     p.total_items = 0;   // the lengths live on the device: every block derives the item list and its range itself
     p.base = 0;
@@ -578,7 +607,7 @@ ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, cons
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
     p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
-    EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<true>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
+    EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<true, false>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
                              static_cast<cudaStream_t>(stream), tmK, tmV, p));
     return EF_OK;
 }

@@ -305,6 +305,27 @@ def test_decode_against_scipy_softmax_and_head_mapping():
     np.testing.assert_allclose(oracle.gqa_decode(Q, K[:, :, perm], V[:, :, perm], scale), o, **TOL)
 
 
+def test_decode_window_and_sinks():
+    """Sliding window + sinks in decode: scipy softmax over the explicitly gathered visible keys; no window (0 or
+    >= L) is the plain program bit for bit; window 1 returns the last value row; sinks add exactly the first keys."""
+    B, Hq, Hkv, L, D = 2, 4, 2, 11, 3
+    Q = RNG.standard_normal((B, Hq, D)); K = RNG.standard_normal((B, Hkv, L, D)); V = RNG.standard_normal((B, Hkv, L, D))
+    scale = 0.45
+    for window, sinks in [(4, 0), (4, 2), (1, 0), (1, 3), (10, 1), (5, 9)]:
+        o = oracle.gqa_decode_window(Q, K, V, scale, window, sinks)
+        idx = [j for j in range(L) if j >= L - window or j < sinks]
+        Kx, Vx = np.repeat(K[:, :, idx], Hq // Hkv, axis=1), np.repeat(V[:, :, idx], Hq // Hkv, axis=1)
+        ref = np.einsum("bhl,bhld->bhd", softmax(np.einsum("bhd,bhld->bhl", Q, Kx) * scale, axis=-1), Vx)
+        np.testing.assert_allclose(o, ref, **TOL)
+    plain = oracle.gqa_decode(Q, K, V, scale)
+    assert np.array_equal(oracle.gqa_decode_window(Q, K, V, scale, 0, 3), plain)
+    assert np.array_equal(oracle.gqa_decode_window(Q, K, V, scale, L, 3), plain)
+    assert np.array_equal(oracle.gqa_decode_window(Q, K, V, scale, L + 7, 0), plain)
+    o1 = oracle.gqa_decode_window(Q, K, V, scale, 1, 0)
+    for h in range(Hq):
+        assert np.array_equal(o1[:, h], V[:, h // 2, L - 1])
+
+
 def test_decode_varlen_against_scipy_softmax_per_entry():
     """Per-sequence lengths: entry b is plain softmax attention over its first len_b keys (library routines on the
     truncated tensors), padding rows are never read (NaN there changes nothing), an entry without keys is zero,

@@ -22,7 +22,7 @@ import numpy as np
 
 PROGRAMS = ("rmsnorm_matmul", "gated_mlp", "gqa_decode", "qknorm_attn", "lora_linear")
 # programs beyond the five benchmark configurations (the "next" rows of the scope table)
-EXTRA_PROGRAMS = ("rmsnorm_gated_mlp", "gqa_decode_varlen", "layernorm_matmul", "qknorm_attn_ex")
+EXTRA_PROGRAMS = ("rmsnorm_gated_mlp", "gqa_decode_varlen", "layernorm_matmul", "qknorm_attn_ex", "gqa_decode_window")
 _PROGRAM_ID = {name: i for i, name in enumerate(PROGRAMS + EXTRA_PROGRAMS)}
 
 
@@ -115,6 +115,10 @@ SHAPES = {
         "full": dict(B=8, Hq=32, Hkv=8, L=4096, D=128, scale=1.0 / np.sqrt(128.0)),
         "small": dict(B=2, Hq=8, Hkv=2, L=333, D=128, scale=1.0 / np.sqrt(128.0)),
     },
+    "gqa_decode_window": {  # one query token over a 32K history: 4 sink tokens + the last 4096 (Section 7.3), batch 8
+        "full": dict(B=8, Hq=32, Hkv=8, L=32768, D=128, scale=1.0 / np.sqrt(128.0), window=4096, sinks=4),
+        "small": dict(B=2, Hq=8, Hkv=2, L=1500, D=128, scale=1.0 / np.sqrt(128.0), window=333, sinks=4),
+    },
     "gqa_decode_varlen": {  # serving batch with a length mix: lengths uniform in [1, L], one full, one of length 1
         "full": dict(B=16, Hq=32, Hkv=8, L=4096, D=128, scale=1.0 / np.sqrt(128.0)),
         "small": dict(B=5, Hq=8, Hkv=2, L=333, D=128, scale=1.0 / np.sqrt(128.0)),
@@ -171,6 +175,13 @@ def make_inputs(program: str, seed: int = 0, size: str = "full", **overrides):
             "W": g(3, (K, N), 0.0, 1.0 / np.sqrt(K)),
         }
     elif program == "gqa_decode":
+        B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
+        t = {
+            "Q": g(0, (B, Hq, D), 0.0, 1.0),
+            "K": g(1, (B, Hkv, L, D), 0.0, 1.0),
+            "V": g(2, (B, Hkv, L, D), 0.0, 1.0),
+        }
+    elif program == "gqa_decode_window":
         B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
         t = {
             "Q": g(0, (B, Hq, D), 0.0, 1.0),
@@ -245,6 +256,11 @@ def algorithmic_work(program: str, p: dict) -> dict:
     if program == "gqa_decode":
         B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
         return dict(flops=4 * B * Hq * L * D, bytes=2 * (2 * B * Hkv * L * D + 2 * B * Hq * D))
+    if program == "gqa_decode_window":   # visible keys only
+        B, Hq, Hkv, L, D = p["B"], p["Hq"], p["Hkv"], p["L"], p["D"]
+        w, sk = p["window"], p["sinks"]
+        vis = L if (w <= 0 or w >= L) else w + min(sk, L - w)
+        return dict(flops=4 * B * Hq * vis * D, bytes=2 * (2 * B * Hkv * vis * D + 2 * B * Hq * D))
     if program == "gqa_decode_varlen":   # needs the lengths: p["lens_sum"] = sum of clamped lengths
         Hq, Hkv, D = p["Hq"], p["Hkv"], p["D"]
         tot = int(p["lens_sum"])

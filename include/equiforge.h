@@ -193,7 +193,7 @@ size_t ef_lora_linear_workspace_bytes(int M, int K, int N, int R);
  * allowed to allocate device memory at the point of the call -- for example code that runs
  * inside a memory pool it must not grow, inside a real-time loop, or under a framework that
  * forbids cudaMalloc after start-up.  Instead of a caller workspace the call uses a scratch
- * array of 2,170,880 bytes that is part of the library image; every GPU that loads the library
+ * array of 2,228,224 bytes that is part of the library image; every GPU that loads the library
  * holds that array until the process exits.
  *   - Limit: B * Hkv <= ef_gqa_decode_static_max_units() (1024); larger problems return
  *     EF_ERR_WORKSPACE and nothing is enqueued.  Other errors as for ef_gqa_decode.
@@ -212,8 +212,11 @@ size_t ef_gqa_decode_static_max_units(void);
 /* ---- Workspace and status -------------------------------------------------------------------
  * (No counterpart in the paper: library plumbing.)
  * ef_workspace_init: enqueue zero-fill of the first min(ws_bytes, 64 KiB) bytes of ws on
- *   `stream` (status word, cross-block arrival counters).  Call once per workspace, and again
- *   after ef_check_status reported EF_ERR_DEVICE_TIMEOUT.
+ *   `stream` (status word, cross-block arrival counters).  Call once per workspace, again after
+ *   ef_check_status reported EF_ERR_DEVICE_TIMEOUT, and before handing the workspace to a
+ *   DIFFERENT entry point (each entry point keeps its own words in that window).  Calls of one
+ *   entry point with different shapes may share a workspace that is large enough for each of them
+ *   (the layout does not depend on the shape); calls that may overlap in time need separate ones.
  * ef_check_status: synchronise `stream`, read the 4-byte status word at ws[0]; returns EF_OK,
  *   EF_ERR_DEVICE_TIMEOUT, or EF_ERR_CUDA if the stream itself failed. */
 ef_status ef_workspace_init(void* ws, size_t ws_bytes, void* stream);

@@ -667,7 +667,7 @@ extern "C" {
 
 size_t ef_qknorm_attn_workspace_bytes(int B, int H, int S, int D) {
     if (B <= 0 || H <= 0 || S <= 0 || D != ef::attn::kD) return 0;
-    return ef::kHeaderBytes + static_cast<size_t>(B) * H * S * D * 2;   // header + Khat (normalised keys, bf16)
+    return ef::kDataOffset + static_cast<size_t>(B) * H * S * D * 2;   // header window + Khat (normalised keys, fp16)
 }
 
 ef_status ef_qknorm_attn_ex(const void* Q, const void* K, const void* V, const void* gamma_q, const void* gamma_k, void* O,
@@ -701,7 +701,7 @@ ef_status ef_qknorm_attn_ex(const void* Q, const void* K, const void* V, const v
     ef_status st;
     if ((st = encode_tmap_bf16(&tmQ, Q, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
     uint8_t* w = static_cast<uint8_t*>(ws);
-    __nv_bfloat16* Khat = reinterpret_cast<__nv_bfloat16*>(w + kHeaderBytes);
+    __nv_bfloat16* Khat = reinterpret_cast<__nv_bfloat16*>(w + kDataOffset);
     if ((st = encode_tmap_bf16(&tmK, Khat, 3, kdims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
     if ((st = encode_tmap_bf16(&tmV, V, 3, kdims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
 

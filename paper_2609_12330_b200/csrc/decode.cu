@@ -476,8 +476,7 @@ extern "C" {
 size_t ef_gqa_decode_workspace_bytes(int B, int Hq, int Hkv, int L, int D) {
     (void)Hq; (void)L; (void)D;
     if (B <= 0 || Hkv <= 0) return 0;
-    const size_t counters = ((static_cast<size_t>(B) * Hkv * sizeof(uint32_t)) + 255) & ~size_t(255);
-    return ef::kHeaderBytes + counters + static_cast<size_t>(ef::decode::kMaxGrid) * 2 * ef::decode::kSlotFloats * sizeof(float);
+    return ef::kDataOffset + static_cast<size_t>(ef::decode::kMaxGrid) * 2 * ef::decode::kSlotFloats * sizeof(float);
 }
 
 ef_status ef_gqa_decode_window(const void* Q, const void* K, const void* V, void* O, int B, int Hq, int Hkv, int L, int D,
@@ -541,7 +540,7 @@ ef_status ef_gqa_decode_window(const void* Q, const void* K, const void* V, void
     uint8_t* w = static_cast<uint8_t*>(ws);
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
-    p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
+    p.partials = reinterpret_cast<float*>(w + kDataOffset);
     if (win_start > 0)
         EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<false, true>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
                                  static_cast<cudaStream_t>(stream), tmK, tmV, p));
@@ -606,7 +605,7 @@ ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, cons
     uint8_t* w = static_cast<uint8_t*>(ws);
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
-    p.partials = reinterpret_cast<float*>(w + kHeaderBytes + counters_bytes);
+    p.partials = reinterpret_cast<float*>(w + kDataOffset);
     EF_CUDA_CHECK(launch_pdl(decode::gqa_decode_kernel<true, false>, dim3(grid), dim3(decode::kThreads), decode::kSmemBytes,
                              static_cast<cudaStream_t>(stream), tmK, tmV, p));
     return EF_OK;
@@ -623,8 +622,7 @@ ef_status ef_gqa_decode_varlen(const void* Q, const void* K, const void* V, cons
 namespace ef {
 namespace decode {
 constexpr int kStaticMaxUnits = 1024;  // B * Hkv accepted by ef_gqa_decode_static
-constexpr size_t kStaticScratchBytes =
-    kHeaderBytes + kStaticMaxUnits * sizeof(uint32_t) + static_cast<size_t>(kMaxGrid) * 2 * kSlotFloats * sizeof(float);
+constexpr size_t kStaticScratchBytes = kDataOffset + static_cast<size_t>(kMaxGrid) * 2 * kSlotFloats * sizeof(float);
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 // On the host, `g_static_scratch` is only a handle for the runtime, not a device address; the
 // address the kernel needs is looked up once per device and cached here.

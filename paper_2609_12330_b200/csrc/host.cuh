@@ -13,6 +13,10 @@ namespace ef {
 constexpr size_t kHeaderBytes = 4096;
 constexpr size_t kCounterOffset = 256;
 constexpr size_t kMaxCounters = (kHeaderBytes - kCounterOffset) / sizeof(uint32_t);  // 960
+// [kHeaderBytes, kDataOffset) holds only words that are zero between calls (per-tile / per-unit arrival counters) and is
+// inside the window ef_workspace_init clears; whatever a call leaves behind non-zero (partial slots, T, Khat) starts at
+// kDataOffset -- at a FIXED offset, so that calls of one entry point with different shapes can share a workspace.
+constexpr size_t kDataOffset = 65536;
 
 extern thread_local int g_last_cuda_error;
 

@@ -1,16 +1,17 @@
 // ef_lora_linear: Y = X @ W + alpha * (X @ A) @ Bm, tensor-core bound at large M.
 //
-// Two kernels, the form the paper's search selects for LoRA (Section 7.2): the low-rank
-// projection is computed once and stored instead of being recomputed per output tile.
-//   1. lora_t_kernel    T = alpha * (X @ A)              [M,16] bf16 in the workspace
-//   2. lora_main_kernel Y = [X | T] @ [W ; Bm]           the rank-16 update is ONE extra K slab
-// Both run on tcgen05: TMA stages 128B-swizzled bf16 tiles in shared memory, one elected thread
-// issues tcgen05.mma (kind::f16, bf16 operands, fp32 accumulators in TMEM), the epilogue warps
-// read the accumulators back with tcgen05.ld.
+// The form the paper's search selects for LoRA (Section 7.2): the low-rank projection T = alpha * (X @ A) is
+// computed ONCE and stored ([M,16] bf16 in the workspace) instead of being recomputed per output tile, and the
+// rank-16 update enters the main contraction as one extra K slab: Y = [X | T] @ [W ; Bm].  Both steps run in one
+// launch: the grid has one block per SM, the blocks that have no output tile (or, if all have one, the last 16)
+// compute T's 128-row pieces first and publish each with a release store; a tile's producer acquires the pieces it
+// needs right before its last k block, ~40 us later on the benchmark shape, so T costs nothing on the critical path.
+// (For M <= 16 the two steps are two launches of the weight-streaming skinny kernel instead.)
+// Everything runs on tcgen05: TMA stages 128B-swizzled bf16 tiles in shared memory, one elected thread issues
+// tcgen05.mma (kind::f16, bf16 operands, fp32 accumulators in TMEM), the epilogue warps read the accumulators back
+// with tcgen05.ld.
 //
-// Refinement (Table 1): kernel 2 is the "MN" row (grid over 128x256 output tiles, K traversed by
-// the in-block loop); kernel 1 is "MK" (K split across blocks, partial products combined by a
-// parallel Reduce_+ in split order by the block that arrives last -- deterministic).
+// Refinement (Table 1): "MN" -- grid over output tiles, K traversed by the in-block loop.
 //
 // Operand layouts.  X tiles are K-major (K contiguous), W / Bm / A tiles are MN-major (N
 // contiguous) exactly as they sit in global memory; the UMMA descriptors carry the major-ness, so
@@ -50,13 +51,24 @@ struct MainParams {
     int tiles_m, num_tiles;
     int k_blocks;   // K / 64
     int has_lora;   // 1: one more K block taken from (T, Bm)
+    // T = alpha * X @ A is computed INSIDE this kernel by its last t_blocks blocks before they take output tiles
+    // (on the benchmark shape those blocks have no tile at all: 128 tiles, 148 SMs), 128 rows at a time; every
+    // finished 128-row piece is published by the last of its four epilogue warps (flags[2*piece]: arrivals, back to
+    // zero; flags[2*piece+1] = epoch + 1), and a tile's producer waits for that value before it loads the T operand
+    // of its last k block.  The last block to leave advances the epoch.
+    int t_blocks, n_sub;       // blocks that compute T first; 128-row pieces of T
+    float alpha;
+    __nv_bfloat16* T;          // [m_pad][16]
+    uint32_t* flags;           // [n_sub][2]
+    uint32_t* epoch;           // [0] epoch, [1] blocks done
     uint32_t* status;
 };
 
 template <int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
-                 const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmB, const MainParams p) {
+                 const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmA, const MainParams p) {
     constexpr int kStages = MainCfg<MT>::kStages, kStageBytes = MainCfg<MT>::kStageBytes, kAccBufs = MainCfg<MT>::kAccBufs;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -81,15 +93,32 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();  // T (previous kernel) and Y of earlier calls: no global access above this line
+    pdl_wait();  // no global access above this line
     const int total_kb = p.k_blocks + p.has_lora;
+    const uint32_t epoch = __ldcg(p.epoch);
+    // this block's share of T: pieces tb, tb + t_blocks, ... (none if it is not one of the last t_blocks blocks)
+    const int tb = static_cast<int>(blockIdx.x) - (static_cast<int>(gridDim.x) - p.t_blocks);
+    constexpr int kTBBytes = kBK * kRank * 2;   // 2 KiB: [64 k][16 r] MN-major, 32B swizzle
 
     if (warp == 0) {
         if (lane == 0) {
             tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmW);
             if (p.has_lora) { tma_prefetch_desc(&tmT); tma_prefetch_desc(&tmB); }
+            tma_prefetch_desc(&tmA);
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
+            if (tb >= 0) {
+                for (int sub = tb; sub < p.n_sub && ok; sub += p.t_blocks) {
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+                        uint8_t* sA = smem + stage * kStageBytes;
+                        mbar_expect_tx(&full[stage], kABytes + kTBBytes);
+                        tma_load_2d(sA, &tmX, &full[stage], kb * kBK, sub * kBM);
+                        tma_load_2d(sA + kABytes, &tmA, &full[stage], 0, kb * kBK);
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
             for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile % p.tiles_m) * (MT * kBM), n0 = (tile / p.tiles_m) * kBN;
                 for (int kb = 0; kb < total_kb; ++kb) {
@@ -104,6 +133,25 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                         for (int j = 0; j < kBN / 64; ++j)
                             tma_load_2d(sB + j * kBAtomBytes, &tmW, &full[stage], n0 + 64 * j, kb * kBK);
                     } else {  // rank-16 slab: columns >= 16 of T and rows >= 16 of Bm are out of bounds -> zero
+                        // the pieces of T this tile reads were written by other blocks of this launch: wait for them
+                        // (bounded), then order the generic-proxy observation before the async-proxy reads
+                        for (int h = 0; h < MT && ok; ++h) {
+                            const int sub = m0 / kBM + h;
+                            if (sub >= p.n_sub) break;
+                            const uint32_t want = epoch + 1u;
+                            const unsigned long long t0 = globaltimer_ns();
+                            uint32_t spins = 0;
+                            while (ld_acquire_u32(&p.flags[2 * sub + 1]) != want) {
+                                if ((++spins & 0xFFu) == 0u && (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs)) {
+                                    *abort_flag = 1u;
+                                    atomicCAS(p.status, 0u, kStatusTimeout | 7u);
+                                    ok = false;
+                                    break;
+                                }
+                            }
+                        }
+                        if (!ok) break;
+                        fence_proxy_async_all();
 #pragma unroll
                         for (int h = 0; h < MT; ++h) tma_load_2d(sA + h * kABytes, &tmT, &full[stage], 0, m0 + h * kBM);
 #pragma unroll
@@ -120,6 +168,29 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             int stage = 0; uint32_t phase = 0;
             int iter = 0;
             bool ok = true;
+            if (tb >= 0) {   // T pieces first: M128 N16 accumulators in the first columns of the accumulator buffer
+                constexpr uint32_t idesc_t = make_idesc_bf16(kBM, kRank, 0, 1);
+                for (int sub = tb; sub < p.n_sub && ok; sub += p.t_blocks, ++iter) {
+                    const int acc = kAccBufs == 2 ? (iter & 1) : 0;
+                    const uint32_t acc_phase = kAccBufs == 2 ? ((iter >> 1) & 1) : (iter & 1);
+                    if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * kBN;
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!mbar_wait(&full[stage], phase, abort_flag, p.status, 3)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sA = smem_u32(smem + stage * kStageBytes);
+                        const uint64_t a_desc = make_smem_desc(sA, 16, 1024, kSwizzle128B);
+                        const uint64_t b_desc = make_smem_desc(sA + kABytes, 16, 256, kSwizzle32B);
+                        for (int kk = 0; kk < kBK / 16; ++kk)  // B advances 16 k-rows of 32 B = 512 B
+                            umma_ss(d_tmem, a_desc + static_cast<uint64_t>(kk * 2), b_desc + static_cast<uint64_t>(kk * 32), idesc_t,
+                                    (kb | kk) != 0 ? 1u : 0u);
+                        umma_commit(&empty[stage]);
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (ok) umma_commit(&acc_full[acc]);
+                }
+            }
             for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++iter) {
                 const int acc = kAccBufs == 2 ? (iter & 1) : 0;
                 const uint32_t acc_phase = kAccBufs == 2 ? ((iter >> 1) & 1) : (iter & 1);
@@ -150,7 +221,46 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     } else {
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
         int iter = 0;
-        for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++iter) {
+        bool live = true;
+        if (tb >= 0) {
+            for (int sub = tb; sub < p.n_sub; sub += p.t_blocks, ++iter) {
+                const int acc = kAccBufs == 2 ? (iter & 1) : 0;
+                const uint32_t acc_phase = kAccBufs == 2 ? ((iter >> 1) & 1) : (iter & 1);
+                if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.status, 4))) { live = false; break; }
+                tc_fence_after();
+                uint32_t r[16];
+                tmem_ld16(tmem_base + acc * kBN + (static_cast<uint32_t>(q * 32) << 16), r);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[acc]);
+                const int row = sub * kBM + q * 32 + lane;   // < m_pad: T is padded to whole pieces
+                uint4 lo, hi;
+                lo.x = pack_bf16x2(p.alpha * __uint_as_float(r[0]), p.alpha * __uint_as_float(r[1]));
+                lo.y = pack_bf16x2(p.alpha * __uint_as_float(r[2]), p.alpha * __uint_as_float(r[3]));
+                lo.z = pack_bf16x2(p.alpha * __uint_as_float(r[4]), p.alpha * __uint_as_float(r[5]));
+                lo.w = pack_bf16x2(p.alpha * __uint_as_float(r[6]), p.alpha * __uint_as_float(r[7]));
+                hi.x = pack_bf16x2(p.alpha * __uint_as_float(r[8]), p.alpha * __uint_as_float(r[9]));
+                hi.y = pack_bf16x2(p.alpha * __uint_as_float(r[10]), p.alpha * __uint_as_float(r[11]));
+                hi.z = pack_bf16x2(p.alpha * __uint_as_float(r[12]), p.alpha * __uint_as_float(r[13]));
+                hi.w = pack_bf16x2(p.alpha * __uint_as_float(r[14]), p.alpha * __uint_as_float(r[15]));
+                uint4* dst = reinterpret_cast<uint4*>(p.T + static_cast<size_t>(row) * kRank);
+                dst[0] = lo; dst[1] = hi;
+                __threadfence();   // the rows are visible before the flag moves
+                __syncwarp();
+                if (lane == 0) {
+                    // the last of the four warps publishes the piece: ready word = epoch + 1 (a word left behind by an
+                    // earlier call, of this or another shape, is at most the current epoch and can never match)
+                    const uint32_t prev = atomicAdd(&p.flags[2 * sub], 1u);
+                    if (prev == 3u) {
+                        p.flags[2 * sub] = 0u;
+                        __threadfence();
+                        st_release_u32(&p.flags[2 * sub + 1], epoch + 1u);
+                    }
+                }
+            }
+        }
+        for (int tile = blockIdx.x; live && tile < p.num_tiles; tile += gridDim.x, ++iter) {
             const int acc = kAccBufs == 2 ? (iter & 1) : 0;
             const uint32_t acc_phase = kAccBufs == 2 ? ((iter >> 1) & 1) : (iter & 1);
             const int m0 = (tile % p.tiles_m) * (MT * kBM), n0 = (tile / p.tiles_m) * kBN;
@@ -194,178 +304,32 @@ lora_main_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-}
-
-// --------------------------------------------------------------------------------------------
-// T kernel: T = alpha * (X @ A), split-K with an ordered last-arriver reduction
-// --------------------------------------------------------------------------------------------
-constexpr int kTStages = 8;
-constexpr int kTBBytes = kBK * kRank * 2;         // 2 KiB: [64 k][16 r] MN-major, 32B swizzle
-constexpr int kTStageBytes = kABytes + kTBBytes;  // 18 KiB
-constexpr int kTThreads = 192;
-constexpr int kTSmemBytes = 1024 + kTStages * kTStageBytes + 256;
-constexpr uint32_t kTTmemCols = 32;
-
-struct TParams {
-    __nv_bfloat16* T;    // [m_pad][16]
-    float* partials;     // [splits][m_pad][16]
-    uint32_t* counters;  // one per m block, zero between calls
-    int M, m_pad, k_blocks, splits;
-    float alpha;
-    uint32_t* status;
-};
-
-__global__ void __launch_bounds__(kTThreads, 1)
-lora_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA, const TParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTStages * kTStageBytes);
-    uint64_t* full = bars;                  // [kTStages]
-    uint64_t* acc_full = bars + kTStages;   // [1]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kTStages + 1);
-    volatile uint32_t* abort_flag = tmem_slot + 1;
-    uint32_t* is_last = tmem_slot + 2;
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m_blk = blockIdx.x, split = blockIdx.y;
-    const int kb_begin = (split * p.k_blocks) / p.splits, kb_end = ((split + 1) * p.k_blocks) / p.splits;
-    const int n_kb = kb_end - kb_begin;  // host guarantees 1 <= n_kb <= kTStages
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kTStages; ++s) mbar_init(&full[s], 1);
-        mbar_init(acc_full, 1);
-        *abort_flag = 0u;
-        *is_last = 0u;
-        fence_mbar_init();
-    }
-    if (warp == 1) { tmem_alloc(tmem_slot, kTTmemCols); tmem_relinquish(); }
-    pdl_launch_dependents();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();
-
-    if (warp == 0) {
-        if (lane == 0) {
-            tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmA);
-            for (int i = 0; i < n_kb; ++i) {  // every k block has its own stage: no reuse, no empty barrier
-                uint8_t* sA = smem + i * kTStageBytes;
-                mbar_expect_tx(&full[i], kTStageBytes);
-                tma_load_2d(sA, &tmX, &full[i], (kb_begin + i) * kBK, m_blk * kBM);
-                tma_load_2d(sA + kABytes, &tmA, &full[i], 0, (kb_begin + i) * kBK);
-            }
+    if (threadIdx.x == 0) {   // the last block to leave opens the next epoch of the T flags
+        __threadfence();
+        const uint32_t prev = atomicAdd(&p.epoch[1], 1u);
+        if (prev == gridDim.x - 1) {
+            p.epoch[1] = 0u;
+            p.epoch[0] = epoch + 1u;
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(kBM, kRank, 0, 1);
-            bool ok = true;
-            for (int i = 0; i < n_kb && ok; ++i) {
-                if (!mbar_wait(&full[i], 0u, abort_flag, p.status, 5)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t sA = smem_u32(smem + i * kTStageBytes);
-                const uint64_t a_desc = make_smem_desc(sA, 16, 1024, kSwizzle128B);
-                const uint64_t b_desc = make_smem_desc(sA + kABytes, 16, 256, kSwizzle32B);
-                for (int kk = 0; kk < kBK / 16; ++kk)  // B advances 16 k-rows of 32 B = 512 B
-                    umma_ss(tmem_base, a_desc + static_cast<uint64_t>(kk * 2), b_desc + static_cast<uint64_t>(kk * 32), idesc,
-                            (i | kk) != 0 ? 1u : 0u);
-            }
-            if (ok) umma_commit(acc_full);
-        }
-    } else {
-        const int q = warp & 3;
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0u, abort_flag, p.status, 6));
-        if (ok) {
-            tc_fence_after();
-            uint32_t r[16];
-            tmem_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16), r);
-            tmem_wait_ld();
-            const int row = m_blk * kBM + q * 32 + lane;  // < m_pad always
-            if (p.splits == 1) {
-                uint4 lo, hi;
-                lo.x = pack_bf16x2(p.alpha * __uint_as_float(r[0]), p.alpha * __uint_as_float(r[1]));
-                lo.y = pack_bf16x2(p.alpha * __uint_as_float(r[2]), p.alpha * __uint_as_float(r[3]));
-                lo.z = pack_bf16x2(p.alpha * __uint_as_float(r[4]), p.alpha * __uint_as_float(r[5]));
-                lo.w = pack_bf16x2(p.alpha * __uint_as_float(r[6]), p.alpha * __uint_as_float(r[7]));
-                hi.x = pack_bf16x2(p.alpha * __uint_as_float(r[8]), p.alpha * __uint_as_float(r[9]));
-                hi.y = pack_bf16x2(p.alpha * __uint_as_float(r[10]), p.alpha * __uint_as_float(r[11]));
-                hi.z = pack_bf16x2(p.alpha * __uint_as_float(r[12]), p.alpha * __uint_as_float(r[13]));
-                hi.w = pack_bf16x2(p.alpha * __uint_as_float(r[14]), p.alpha * __uint_as_float(r[15]));
-                uint4* dst = reinterpret_cast<uint4*>(p.T + static_cast<size_t>(row) * kRank);
-                dst[0] = lo; dst[1] = hi;
-            } else {
-                uint4* dst = reinterpret_cast<uint4*>(p.partials + (static_cast<size_t>(split) * p.m_pad + row) * kRank);
-                dst[0] = make_uint4(r[0], r[1], r[2], r[3]);
-                dst[1] = make_uint4(r[4], r[5], r[6], r[7]);
-                dst[2] = make_uint4(r[8], r[9], r[10], r[11]);
-                dst[3] = make_uint4(r[12], r[13], r[14], r[15]);
-                __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (warp == 2 && lane == 0) {
-                    const uint32_t prev = atomicAdd(&p.counters[m_blk], 1u);
-                    *is_last = (prev == static_cast<uint32_t>(p.splits - 1)) ? 1u : 0u;
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (*is_last) {
-                    __threadfence();
-                    float acc[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-                    for (int s = 0; s < p.splits; ++s) {  // split order: deterministic
-                        const float4* src = reinterpret_cast<const float4*>(p.partials + (static_cast<size_t>(s) * p.m_pad + row) * kRank);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float4 v = __ldcg(src + j);
-                            acc[4 * j] += v.x; acc[4 * j + 1] += v.y; acc[4 * j + 2] += v.z; acc[4 * j + 3] += v.w;
-                        }
-                    }
-                    uint4 lo, hi;
-                    lo.x = pack_bf16x2(p.alpha * acc[0], p.alpha * acc[1]);
-                    lo.y = pack_bf16x2(p.alpha * acc[2], p.alpha * acc[3]);
-                    lo.z = pack_bf16x2(p.alpha * acc[4], p.alpha * acc[5]);
-                    lo.w = pack_bf16x2(p.alpha * acc[6], p.alpha * acc[7]);
-                    hi.x = pack_bf16x2(p.alpha * acc[8], p.alpha * acc[9]);
-                    hi.y = pack_bf16x2(p.alpha * acc[10], p.alpha * acc[11]);
-                    hi.z = pack_bf16x2(p.alpha * acc[12], p.alpha * acc[13]);
-                    hi.w = pack_bf16x2(p.alpha * acc[14], p.alpha * acc[15]);
-                    uint4* dst2 = reinterpret_cast<uint4*>(p.T + static_cast<size_t>(row) * kRank);
-                    dst2[0] = lo; dst2[1] = hi;
-                    if (warp == 2 && lane == 0) p.counters[m_blk] = 0u;
-                }
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc(tmem_base, kTTmemCols);
     }
 }
 
 struct Plan {
-    int tiles_m, tiles_n, m_pad, k_blocks, splits;
-    size_t t_off, part_off, tail_counters_off, tail_part_off, total;
+    int tiles_m, tiles_n, m_pad, k_blocks;
+    size_t t_off, tail_counters_off, tail_part_off, total;
 };
-inline Plan make_plan(int M, int K, int N, int num_sms) {
+inline Plan make_plan(int M, int K, int N) {
     Plan pl;
     pl.tiles_m = (M + kBM - 1) / kBM;
     pl.tiles_n = (N + kBN - 1) / kBN;
     pl.m_pad = pl.tiles_m * kBM;
     pl.k_blocks = K / kBK;
-    int s = num_sms / pl.tiles_m;
-    if (s < 1) s = 1;
-    if (s > pl.k_blocks) s = pl.k_blocks;
-    const int min_s = (pl.k_blocks + kTStages - 1) / kTStages;  // each split fits the stage ring
-    if (s < min_s) s = min_s;
-    pl.splits = s;
-    // M <= 16 takes the skinny-M second kernel: its per-n-tile arrival counters sit right behind the header (inside
-    // the window ef_workspace_init clears), its partial slots at the end
+    // M <= 16 takes the skinny-M kernels: their per-n-tile arrival counters sit right behind the header (inside
+    // the window ef_workspace_init clears), their partial slots at the end
     const bool skinny_tail = M <= skinny::kLoraTailMaxM;
     pl.tail_counters_off = kHeaderBytes;
-    pl.t_off = kHeaderBytes + (skinny_tail ? skinny::lora_tail_counters_bytes(N) : 0);
-    pl.part_off = pl.t_off + ((static_cast<size_t>(pl.m_pad) * kRank * 2 + 255) & ~size_t(255));
-    pl.tail_part_off = pl.part_off + static_cast<size_t>(pl.k_blocks) * pl.m_pad * kRank * 4;  // worst case: one split per k block
+    pl.t_off = kDataOffset;   // fixed: a workspace may serve calls of different shapes
+    pl.tail_part_off = pl.t_off + ((static_cast<size_t>(pl.m_pad) * kRank * 2 + 255) & ~size_t(255));
     pl.total = pl.tail_part_off + (skinny_tail ? skinny::lora_tail_partials_bytes() : 0);
     return pl;
 }
@@ -377,7 +341,7 @@ extern "C" {
 
 size_t ef_lora_linear_workspace_bytes(int M, int K, int N, int R) {
     if (M <= 0 || K <= 0 || N <= 0 || R != ef::lora::kRank || K % ef::lora::kBK != 0) return 0;
-    return ef::lora::make_plan(M, K, N, 1).total;
+    return ef::lora::make_plan(M, K, N).total;
 }
 
 ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void* Bm, void* Y, int M, int K, int N, int R,
@@ -386,14 +350,14 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
     if (!X || !W || !A || !Bm || !Y) return EF_ERR_NULL;
     if (M <= 0 || K <= 0 || N <= 0 || R <= 0) return EF_ERR_SHAPE;
     if (R != lora::kRank || K % lora::kBK != 0 || N % 8 != 0) return EF_ERR_UNSUPPORTED;
-    if ((M + lora::kBM - 1) / lora::kBM > static_cast<int>(kMaxCounters)) return EF_ERR_UNSUPPORTED;
+    if (2 * ((M + lora::kBM - 1) / lora::kBM) > static_cast<int>(kMaxCounters)) return EF_ERR_UNSUPPORTED;
     if (!aligned(X, 16) || !aligned(W, 16) || !aligned(A, 16) || !aligned(Bm, 16) || !aligned(Y, 16)) return EF_ERR_ALIGN;
     if (!ws || ws_bytes < ef_lora_linear_workspace_bytes(M, K, N, R)) return EF_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return EF_ERR_ALIGN;
     DeviceInfo di;
     if (!current_device_info(&di)) return EF_ERR_CUDA;
     if (di.cc_major != 10) return EF_ERR_ARCH;
-    const lora::Plan pl = lora::make_plan(M, K, N, di.num_sms);
+    const lora::Plan pl = lora::make_plan(M, K, N);
     uint8_t* w = static_cast<uint8_t*>(ws);
     __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(w + pl.t_off);
 
@@ -433,30 +397,18 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
     if (!attr_set[di.device]) {
         EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_main_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::MainCfg<1>::kSmemBytes));
         EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_main_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::MainCfg<2>::kSmemBytes));
-        EF_CUDA_CHECK(cudaFuncSetAttribute(lora::lora_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lora::kTSmemBytes));
         attr_set[di.device] = true;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (M <= skinny::kLoraTailMaxM) {
         // Few rows: both kernels are weight-streaming problems, not tensor-bound ones.  Same two-kernel form
         // (T stored once, reused by every output tile), on the skinny-projection kernel.
-        if (pl.t_off > 65536) return EF_ERR_UNSUPPORTED;   // counters must lie in the init window
+        if (kHeaderBytes + skinny::lora_tail_counters_bytes(N) > kDataOffset) return EF_ERR_UNSUPPORTED;   // counters must lie in the init window
         uint32_t* status = reinterpret_cast<uint32_t*>(w);
         uint32_t* counters = reinterpret_cast<uint32_t*>(w + pl.tail_counters_off);
         float* partials = reinterpret_cast<float*>(w + pl.tail_part_off);
         if ((st = skinny::launch_lora_head(X, A, T, M, K, alpha, status, counters, partials, di, s)) != EF_OK) return st;
         return skinny::launch_lora_tail(X, W, T, Bm, Y, M, K, N, status, counters, partials, di, s);
-    }
-    {
-        lora::TParams tp;
-        tp.T = T;
-        tp.partials = reinterpret_cast<float*>(w + pl.part_off);
-        tp.counters = reinterpret_cast<uint32_t*>(w + kCounterOffset);
-        tp.M = M; tp.m_pad = pl.m_pad; tp.k_blocks = pl.k_blocks; tp.splits = pl.splits;
-        tp.alpha = alpha;
-        tp.status = reinterpret_cast<uint32_t*>(w);
-        EF_CUDA_CHECK(launch_pdl(lora::lora_t_kernel, dim3(pl.tiles_m, pl.splits), dim3(lora::kTThreads), lora::kTSmemBytes, s,
-                                 tmX, tmA, tp));
     }
     {
         lora::MainParams mp;
@@ -470,13 +422,24 @@ ef_status ef_lora_linear(const void* X, const void* W, const void* A, const void
         mp.num_tiles = mp.tiles_m * pl.tiles_n;
         mp.k_blocks = pl.k_blocks; mp.has_lora = 1;
         mp.status = reinterpret_cast<uint32_t*>(w);
-        const int grid = di.num_sms < mp.num_tiles ? di.num_sms : mp.num_tiles;
+        // T = alpha * X @ A inside the same launch: the grid always has #SMs blocks (all resident at once, one per
+        // SM), and the last t_blocks of them compute T's 128-row pieces before they look for output tiles.
+        mp.alpha = alpha;
+        mp.T = T;
+        mp.flags = reinterpret_cast<uint32_t*>(w + kCounterOffset);
+        mp.epoch = reinterpret_cast<uint32_t*>(w + 64);
+        mp.n_sub = pl.tiles_m;
+        const int grid = di.num_sms;
+        int idle = grid - mp.num_tiles;
+        if (idle < 0) idle = 0;
+        mp.t_blocks = idle >= 4 ? idle : (grid < 16 ? grid : 16);   // idle blocks if there are some, else the last 16
+        if (mp.t_blocks > mp.n_sub) mp.t_blocks = mp.n_sub;
         if (mt == 2)
             EF_CUDA_CHECK(launch_pdl(lora::lora_main_kernel<2>, dim3(grid), dim3(lora::kThreads), lora::MainCfg<2>::kSmemBytes, s,
-                                     tmX, tmW, tmT, tmB, mp));
+                                     tmX, tmW, tmT, tmB, tmA, mp));
         else
             EF_CUDA_CHECK(launch_pdl(lora::lora_main_kernel<1>, dim3(grid), dim3(lora::kThreads), lora::MainCfg<1>::kSmemBytes, s,
-                                     tmX, tmW, tmT, tmB, mp));
+                                     tmX, tmW, tmT, tmB, tmA, mp));
     }
     return EF_OK;
 }

@@ -433,7 +433,7 @@ inline bool make_plan(int NW, bool norm, int K, int N, Plan* pl) {
     pl->stages = stages;
     pl->smem_bytes = 1024 + xg + stages * pl->stage_bytes + kMiscBytes;
     pl->counters_bytes = (static_cast<size_t>(pl->n_tiles) * 4 + 255) & ~size_t(255);
-    pl->total = kHeaderBytes + pl->counters_bytes + static_cast<size_t>(kMaxGrid) * 2 * NW * kMaxM * kBN * 4;
+    pl->total = kDataOffset + static_cast<size_t>(kMaxGrid) * 2 * NW * kMaxM * kBN * 4;
     return stages >= 2;
 }
 
@@ -501,7 +501,7 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
     uint8_t* w = static_cast<uint8_t*>(ws);
     p.status = reinterpret_cast<uint32_t*>(w);
     p.counters = reinterpret_cast<uint32_t*>(w + kHeaderBytes);
-    p.partials = reinterpret_cast<float*>(w + kHeaderBytes + pl.counters_bytes);
+    p.partials = reinterpret_cast<float*>(w + kDataOffset);
     EF_CUDA_CHECK(launch_pdl(skinny_kernel<NW, NORM>, dim3(grid), dim3(kThreads), static_cast<size_t>(pl.smem_bytes),
                              static_cast<cudaStream_t>(stream), tmW0, tmW1, tmX, tmX, p));
     return EF_OK;

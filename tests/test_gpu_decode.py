@@ -64,3 +64,28 @@ def test_decode_peaky_logits():
 def test_decode_full_config():
     r = _run(0, size="full")
     assert r["rel_l2"] < 5e-3
+
+
+def test_one_workspace_serves_calls_of_different_shapes():
+    import torch
+
+    import oracle
+    import paper_2609_12330_b200 as ef
+    import workloads as wl
+    from parity import assert_close
+
+    shapes = [dict(B=1, Hq=8, Hkv=2, L=700), dict(B=40, Hq=8, Hkv=8, L=333), dict(B=2, Hq=8, Hkv=1, L=5000),
+              dict(B=40, Hq=8, Hkv=8, L=333)]
+    cases, need = [], 0
+    for i, sh in enumerate(shapes):
+        p, t = wl.make_inputs("gqa_decode", seed=40 + i, size="small", **sh)
+        cases.append((p, t))
+        need = max(need, ef.workspace_bytes("gqa_decode", p))
+    ws = ef.Workspace(need)
+    for p, t in cases:
+        dev = {k: wl.to_torch(k, v, "cuda") for k, v in t.items()}
+        ref = oracle.run("gqa_decode", p, {k: wl.to_f64(k, v) for k, v in t.items()})
+        out = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        ef.run("gqa_decode", p, dev, ws, out=out)
+        ws.check()
+        assert_close(wl.torch_bf16_to_f64(out), ref, f"gqa_decode {p}")

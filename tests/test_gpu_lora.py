@@ -57,3 +57,33 @@ def test_lora_256_row_block_tiles(M, K, N):
     # enough 128x256 tiles for two waves of the grid: the kernel instance with 256-row block tiles runs,
     # with ragged rows in the last tile and a ragged last column tile
     run_parity("lora_linear", seed=10, size="small", M=M, K=K, N=N, check_repeat=False)
+
+
+def test_lora_workspace_reused_across_shapes_and_calls():
+    """One workspace, calls of different shapes in a row: the in-kernel hand-over of T (per-piece ready words keyed by
+    an epoch) must not be confused by words a differently shaped earlier call left behind."""
+    import numpy as np
+    import torch
+
+    import oracle
+    import paper_2609_12330_b200 as ef
+    import workloads as wl
+    from parity import assert_close
+
+    shapes = [dict(M=256, K=128, N=264), dict(M=700, K=192, N=520), dict(M=130, K=64, N=256), dict(M=700, K=192, N=520),
+              dict(M=9, K=128, N=264), dict(M=512, K=256, N=9728), dict(M=256, K=128, N=264)]
+    need = 0
+    cases = []
+    for i, sh in enumerate(shapes):
+        p, t = wl.make_inputs("lora_linear", seed=20 + i, size="small", **sh)
+        need = max(need, ef.workspace_bytes("lora_linear", p))
+        cases.append((p, t))
+    ws = ef.Workspace(need)
+    for p, t in cases:
+        dev = {k: wl.to_torch(k, v, "cuda") for k, v in t.items()}
+        ref = oracle.run("lora_linear", p, {k: wl.to_f64(k, v) for k, v in t.items()})
+        for _ in range(2):
+            out = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+            ef.run("lora_linear", p, dev, ws, out=out)
+            ws.check()
+            assert_close(wl.torch_bf16_to_f64(out), ref, f"lora {p}")

@@ -76,3 +76,30 @@ def test_rmsnorm_gated_mlp_shapes(M, K, N):
 def test_rmsnorm_gated_mlp_full_config():
     r = run_parity("rmsnorm_gated_mlp", 0, size="full")   # batch 8, 4096 -> 11008
     assert r["rel_l2"] < 5e-3
+
+
+def test_one_workspace_serves_calls_of_different_shapes():
+    """The workspace layout does not depend on the shape: a small-N call must not leave partial sums where a later
+    large-N call keeps its arrival counters."""
+    import torch
+
+    import oracle
+    import paper_2609_12330_b200 as ef
+    import workloads as wl
+    from parity import assert_close
+
+    shapes = [dict(M=5, K=192, N=136), dict(M=16, K=1024, N=11008), dict(M=3, K=64, N=8), dict(M=16, K=1024, N=11008),
+              dict(M=9, K=4096, N=1000)]
+    cases, need = [], 0
+    for i, sh in enumerate(shapes):
+        p, t = wl.make_inputs("gated_mlp", seed=30 + i, size="small", **sh)
+        cases.append((p, t))
+        need = max(need, ef.workspace_bytes("gated_mlp", p))
+    ws = ef.Workspace(need)
+    for p, t in cases:
+        dev = {k: wl.to_torch(k, v, "cuda") for k, v in t.items()}
+        ref = oracle.run("gated_mlp", p, {k: wl.to_f64(k, v) for k, v in t.items()})
+        out = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        ef.run("gated_mlp", p, dev, ws, out=out)
+        ws.check()
+        assert_close(wl.torch_bf16_to_f64(out), ref, f"gated_mlp {p}")

@@ -33,7 +33,7 @@ METRIC = "us/call and TFLOP/s (GB/s for decode) per fused program, % of B200 roo
 UNIT = "TFLOP/s (algorithmic flops of one step = all five programs / step time; per-program us/call, TFLOP/s, GB/s in 'programs')"
 BOUND = {"rmsnorm_matmul": "hbm", "gated_mlp": "hbm", "gqa_decode": "hbm", "qknorm_attn": "tensor", "lora_linear": "tensor",
          "rmsnorm_gated_mlp": "hbm", "gqa_decode_varlen": "hbm", "layernorm_matmul": "hbm", "qknorm_attn_ex": "tensor", "gqa_decode_window": "hbm"}
-KERNELS_PER_CALL = {"rmsnorm_matmul": 1, "gated_mlp": 1, "gqa_decode": 1, "qknorm_attn": 2, "lora_linear": 2,
+KERNELS_PER_CALL = {"rmsnorm_matmul": 1, "gated_mlp": 1, "gqa_decode": 1, "qknorm_attn": 2, "lora_linear": 1,
                     "rmsnorm_gated_mlp": 1, "gqa_decode_varlen": 1, "layernorm_matmul": 1, "qknorm_attn_ex": 2, "gqa_decode_window": 1}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 

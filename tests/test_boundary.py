@@ -61,6 +61,18 @@ def test_host_side_argument_validation(lib):
     assert lib.ef_gqa_decode_varlen(one, one, one, one, one, 1025, 4, 1, 8, 128, 1.0, one, 1 << 30, null) == 3   # B > 1024
     assert lib.ef_gqa_decode_varlen(one, one, one, p(4098), one, 1, 4, 1, 8, 128, 1.0, one, 1 << 30, null) == 4
     assert lib.ef_gqa_decode_varlen(one, one, one, one, one, 1, 4, 1, 8, 128, 1.0, one, 16, null) == 5
+    # windowed decode, LayerNorm projection, attention with grouped heads / window / sinks
+    assert lib.ef_gqa_decode_window(one, one, one, null, 1, 4, 1, 8, 128, 1.0, 4, 0, one, 1 << 30, null) == 1
+    assert lib.ef_gqa_decode_window(one, one, one, one, 1, 4, 1, 8, 128, 1.0, -1, 0, one, 1 << 30, null) == 2
+    assert lib.ef_gqa_decode_window(one, one, one, one, 1, 4, 1, 8, 64, 1.0, 4, 0, one, 1 << 30, null) == 3
+    assert lib.ef_layernorm_matmul(one, one, null, one, one, 4, 64, 8, 1e-5, one, 1 << 30, null) == 1      # beta missing
+    assert lib.ef_layernorm_matmul(one, one, one, one, one, 16, 64, 8, 1e-5, one, 1 << 30, null) == 3       # M > 15
+    assert lib.ef_layernorm_matmul(one, one, one, one, one, 4, 60, 8, 1e-5, one, 1 << 30, null) == 3        # K % 64
+    assert lib.ef_qknorm_attn_ex(one, one, one, one, one, null, 1, 4, 2, 64, 128, 1e-6, 1.0, 1, 0, 0, one, 1 << 30, null) == 1
+    assert lib.ef_qknorm_attn_ex(one, one, one, one, one, one, 1, 5, 2, 64, 128, 1e-6, 1.0, 1, 0, 0, one, 1 << 30, null) == 2   # Hq % Hkv
+    assert lib.ef_qknorm_attn_ex(one, one, one, one, one, one, 1, 4, 2, 64, 128, 1e-6, 1.0, 0, 16, 0, one, 1 << 30, null) == 3  # window, not causal
+    assert lib.ef_qknorm_attn_ex(one, one, one, one, one, one, 1, 4, 2, 64, 128, 1e-6, 1.0, 1, 16, 200, one, 1 << 30, null) == 3  # sinks > 128
+    assert lib.ef_qknorm_attn_ex(one, one, one, one, one, one, 1, 4, 2, 64, 128, 1e-6, 0.0, 1, 0, 0, one, 1 << 30, null) == 3   # scale <= 0
     assert lib.ef_workspace_init(null, 4096, null) == 1
     assert lib.ef_workspace_init(one, 16, null) == 5
 

@@ -401,7 +401,11 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 for (int j = 0; j < g.n_kv && ok; ++j) {
                     const uint32_t nv = 2 * (kv_use + j) + 1, nk = nv + 1;   // load numbers of V_j and K_j+1
                     const uint32_t st = nv % kKVSlots, stn = nk % kKVSlots;
-                    bool v_waited = false, k_waited = false;
+                    // The K/V tiles of this step landed long ago: look at their barriers now, while the softmax groups
+                    // are still busy, so that nothing but the MMAs follows a group's hand-over on the critical path.
+                    if (!mbar_wait(&kv_full[st], (nv / kKVSlots) & 1, abort_flag, p.status, 7)) { ok = false; break; }
+                    if (j + 1 < g.n_kv && !mbar_wait(&kv_full[stn], (nk / kKVSlots) & 1, abort_flag, p.status, 8)) { ok = false; break; }
+                    bool v_waited = true, k_waited = j + 1 < g.n_kv;
                     for (int t = 0; t < 2 && ok; ++t) {
                         if (g.part(t, j)) {
                             if (!mbar_wait(&p_full[t], cp[t] & 1, abort_flag, p.status, 6)) { ok = false; break; }

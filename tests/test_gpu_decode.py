@@ -56,6 +56,13 @@ def test_decode_long_single_unit():
     _run(6, B=1, Hq=4, Hkv=1, L=20000)  # one unit spread over every block: cross-block merge
 
 
+@pytest.mark.parametrize("B,L", [(1, 4096), (2, 4000), (3, 4096), (4, 2500), (12, 1100), (18, 4096)])
+def test_decode_blocks_per_unit_choices(B, L):
+    """The grid is chosen per shape: with no more (batch, kv head) units than SMs every unit gets the same number of
+    blocks (1 ... 18 here; the chunk count is not always a multiple of it), with more units equal chunk ranges."""
+    _run(8, B=B, Hq=32, Hkv=8, L=L)
+
+
 def test_decode_peaky_logits():
     # large scale -> near one-hot softmax; exercises the running-max repair
     _run(7, L=500, scale=4.0)

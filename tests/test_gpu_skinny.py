@@ -23,6 +23,12 @@ def test_gated_mlp_more_units_than_sms():
     run_parity("gated_mlp", 4, M=16, K=512, N=4096)   # 32 tiles x 8 k blocks = 256 units
 
 
+def test_gated_mlp_one_block_per_whole_tile():
+    # 86 n tiles (the last one ragged: 120 columns) x 16 k blocks: enough tiles to saturate HBM with one block each,
+    # so no block shares a tile and no partial results are exchanged
+    run_parity("gated_mlp", 5, M=16, K=1024, N=11000)
+
+
 def test_gated_mlp_full_config():
     r = run_parity("gated_mlp", 0, size="full")
     assert r["rel_l2"] < 5e-3

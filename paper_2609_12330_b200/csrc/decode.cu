@@ -165,15 +165,22 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (warp == 0) {
             const int per = (p.B + 31) / 32;
             const int b0 = lane * per;
-            int sum = 0;
+            int sum = 0, longest = 0;   // items of this lane's entries; most items of one entry
             for (int i = 0; i < per; ++i) {
                 const int b = b0 + i;
                 if (b < p.B) {
                     int len = p.seq_lens[b];
                     len = len < 0 ? 0 : (len > p.L ? p.L : len);
                     cum[p.B + 3 + b] = len;
-                    sum += len > 0 ? (len + kChunk - 1) / kChunk + 1 : 0;
+                    const int items = len > 0 ? (len + kChunk - 1) / kChunk + 1 : 0;
+                    sum += items;
+                    longest = longest > items ? longest : items;
                 }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const int v = __shfl_xor_sync(0xffffffffu, longest, o);
+                longest = longest > v ? longest : v;
             }
             int incl = sum;
 #pragma unroll
@@ -194,6 +201,11 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 const int total = incl * p.Hkv;
                 cum[p.B + 1] = total / static_cast<int>(gridDim.x);
                 cum[p.B + 2] = total % static_cast<int>(gridDim.x);
+                // One block per whole (batch, kv head) unit needs no partial states and no merging block; it wins unless one
+                // sequence is much longer than the average block's share (cost model from measurements: a block alone
+                // streams a chunk in ~0.75 us, all blocks together one in ~0.0115 us, the partial exchange costs ~9 us
+                // with a length mix): every block takes this decision from the same numbers.
+                cum[2 * p.B + 3] = (p.B * p.Hkv <= static_cast<int>(gridDim.x) && longest < total / 65 + 12) ? 1 : 0;
             }
         }
         __syncthreads();
@@ -209,8 +221,17 @@ gqa_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             }
         }
     }
-    const int it_begin = range_begin(blockIdx.x, base, rem);
-    const int it_end = range_begin(blockIdx.x + 1, base, rem);
+    int it_begin = range_begin(blockIdx.x, base, rem);
+    int it_end = range_begin(blockIdx.x + 1, base, rem);
+    if (VARLEN && cum[2 * p.B + 3]) {   // block = unit: every unit is whole, so the merge path below is never entered
+        const int bb = static_cast<int>(blockIdx.x) / p.Hkv, kvh = static_cast<int>(blockIdx.x) - bb * p.Hkv;
+        it_begin = it_end = 0;
+        if (bb < p.B) {
+            const int nb = cum[bb + 1] - cum[bb];
+            it_begin = p.Hkv * cum[bb] + kvh * nb;
+            it_end = it_begin + nb;
+        }
+    }
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer warp ------------------------------

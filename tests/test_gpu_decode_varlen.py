@@ -68,5 +68,16 @@ def test_many_short_sequences():
     run_parity("gqa_decode_varlen", seed=7, size="small", B=200, Hq=8, Hkv=2, L=96)
 
 
+@pytest.mark.parametrize("lens", [
+    [6000, 40, 900],          # one sequence far longer than a block's share: equal ranges, units split and merged
+    [5000, 5000, 5000],       # long and even: split as well (few units)
+    [1500, 700, 1, 0],        # short enough for one block per whole unit
+])
+def test_both_partitions(lens):
+    """The kernel decides from the lengths whether every block takes one whole (batch, kv head) unit or the item list is
+    cut into equal ranges with partial states merged across blocks."""
+    run_parity("gqa_decode_varlen", seed=8, size="small", B=len(lens), L=6016, lens=lens)
+
+
 def test_full_serving_batch():
     run_parity("gqa_decode_varlen", seed=0, size="full")

@@ -43,6 +43,10 @@ struct Params {
     int base, rem;       // block c owns base + (c < rem) consecutive (tile, k block) units
     int stages;
     int lora;            // NW == 1, no norm: the last k block of every n tile is the rank-16 update (T, Bm tiles)
+    int pdl_mode;        // programmatic dependent launch: 0 = let the next kernel start at once, wait for the previous one
+                         // before the first global access; 1 = wait first, THEN let the next kernel start (so the next one
+                         // may read this kernel's inputs without waiting); 2 = no wait except before the T tile is loaded
+                         // (the kernel before is a mode-1 kernel that produces nothing else this one reads)
     float eps;
     float out_scale;     // NW == 1, no norm: the result is multiplied by this before rounding (1 elsewhere)
     uint32_t* status;
@@ -126,12 +130,13 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
         fence_mbar_init();
     }
     if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
-    pdl_launch_dependents();
+    if (p.pdl_mode != 1) pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();  // everything below may touch global memory of the previous kernel in the stream
+    if (p.pdl_mode != 2) pdl_wait();  // everything below may touch global memory of the previous kernel in the stream
+    if (p.pdl_mode == 1) pdl_launch_dependents();
 
     // The producer starts streaming W right away; everyone else first builds the X operand.
     if (warp == 0) {
@@ -142,6 +147,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
             if (NW == 1 && !NORM && p.lora) { tma_prefetch_desc(&tmW1); tma_prefetch_desc(&tmT); }
             int stage = 0; uint32_t phase = 0;
             bool okp = true;
+            bool t_waited = false;
             for (int sg = 0; sg < nseg && okp; ++sg) {
               const Seg seg = seg_of(sg, nseg, it_begin, it_end, p.k_blocks);
               const int tile = seg.it0 / p.k_blocks;
@@ -154,6 +160,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                 if (NW == 1 && !NORM && p.lora && kb == p.k_blocks - 1) {
                     // the rank-16 update as one more k block: Bm rows 16..63 and T columns 16..63 lie outside
                     // their tensors and are filled with zeros (the second weight map carries Bm here)
+                    if (p.pdl_mode == 2 && !t_waited) { pdl_wait(); t_waited = true; }   // T comes from the kernel before
                     tma_load_2d(st, &tmW1, &full[stage], n0, 0);
                     tma_load_2d(st + kWAtomBytes, &tmW1, &full[stage], n0 + 64, 0);
                     tma_load_2d(st + NW * kWBytes, &tmT, &full[stage], 0, 0);
@@ -481,6 +488,7 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.M = M; p.K = K; p.N = N;
     p.lora = 0;
+    p.pdl_mode = 0;
     p.out_scale = 1.f;
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
     int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
@@ -521,10 +529,12 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
 //   launch_lora_head: T = alpha * X @ A   (A is a [K,16] weight: one n tile; few blocks, so few partials to merge)
 //   launch_lora_tail: Y = [X | T] @ [W ; Bm], the rank-16 update as one extra k block.
 size_t lora_tail_counters_bytes(int N) { return 256 + ((static_cast<size_t>((N + kBN - 1) / kBN) * 4 + 255) & ~size_t(255)); }
-size_t lora_tail_partials_bytes() { return static_cast<size_t>(kMaxGrid) * 2 * kMaxM * kBN * 4; }
+constexpr int kLoraHeadGrid = 8;   // one n tile of 16 live columns, K / 64 k blocks: 8 blocks keep the ordered merge short
+// partial slots of the head kernel (kLoraHeadGrid blocks) followed by those of the tail kernel: the two run concurrently
+size_t lora_tail_partials_bytes() { return static_cast<size_t>(kLoraHeadGrid + kMaxGrid) * 2 * kMaxM * kBN * 4; }
 static ef_status launch_plain(const void* X, const void* W, int w_rows, const void* T, const void* Bm, void* Y, int M, int K,
-                              int N, float out_scale, int grid_cap, uint32_t* status, uint32_t* counters, float* partials,
-                              const DeviceInfo& di, cudaStream_t stream) {
+                              int N, float out_scale, int grid_cap, int pdl_mode, uint32_t* status, uint32_t* counters,
+                              float* partials, const DeviceInfo& di, cudaStream_t stream) {
     const bool lora = T != nullptr;
     Plan pl;
     if (M > kMaxM || K % kBK != 0 || N % 8 != 0) return EF_ERR_UNSUPPORTED;
@@ -557,6 +567,7 @@ static ef_status launch_plain(const void* X, const void* W, int w_rows, const vo
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.M = M; p.K = K; p.N = N;
     p.lora = lora ? 1 : 0;
+    p.pdl_mode = pdl_mode;
     p.out_scale = out_scale;
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
     int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
@@ -575,12 +586,14 @@ static ef_status launch_plain(const void* X, const void* W, int w_rows, const vo
 }
 ef_status launch_lora_head(const void* X, const void* A, void* T, int M, int K, float alpha, uint32_t* status,
                            uint32_t* counters, float* partials, const DeviceInfo& di, cudaStream_t stream) {
-    // one n tile of 16 live columns, K / 64 k blocks: 8 blocks keep the ordered merge short
-    return launch_plain(X, A, K, nullptr, nullptr, T, M, K, 16, alpha, 8, status, counters, partials, di, stream);
+    // Waits for the kernel before it and only then lets the tail kernel start: the tail may then read X, W and Bm at once
+    // and stream the weights while T is still being computed here.
+    return launch_plain(X, A, K, nullptr, nullptr, T, M, K, 16, alpha, kLoraHeadGrid, 1, status, counters, partials, di, stream);
 }
 ef_status launch_lora_tail(const void* X, const void* W, const void* T, const void* Bm, void* Y, int M, int K, int N,
                            uint32_t* status, uint32_t* counters, float* partials, const DeviceInfo& di, cudaStream_t stream) {
-    return launch_plain(X, W, K, T, Bm, Y, M, K, N, 1.f, kMaxGrid, status, counters + 64, partials, di, stream);
+    return launch_plain(X, W, K, T, Bm, Y, M, K, N, 1.f, kMaxGrid, 2, status, counters + 64,
+                        partials + static_cast<size_t>(kLoraHeadGrid) * 2 * kMaxM * kBN, di, stream);
 }
 
 }  // namespace skinny

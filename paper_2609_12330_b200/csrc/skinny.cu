@@ -43,6 +43,8 @@ struct Params {
     int base, rem;       // block c owns base + (c < rem) consecutive (tile, k block) units
     int stages;
     int lora;            // NW == 1, no norm: the last k block of every n tile is the rank-16 update (T, Bm tiles)
+    int pair;            // 1: a stage holds TWO consecutive k blocks (weight boxes of 128 rows, 16 KiB each: the copy engine
+                         // moves more per request); only when every range starts at an even k block and has even length
     int pdl_mode;        // programmatic dependent launch: 0 = let the next kernel start at once, wait for the previous one
                          // before the first global access; 1 = wait first, THEN let the next kernel start (so the next one
                          // may read this kernel's inputs without waiting); 2 = no wait except before the T tile is loaded
@@ -100,7 +102,8 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
     const int xg_bytes = NORM ? p.k_blocks * kXBytes : 0;
     uint8_t* xg = smem;                                // NORM: [k_blocks][2 KiB] persistent X operand
     uint8_t* stages = smem + xg_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(stages + p.stages * kStageBytes);
+    const int stage_bytes = p.pair ? 2 * kStageBytes : kStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stages + p.stages * stage_bytes);
     uint64_t* full = bars;                             // [stages]
     uint64_t* empty = bars + p.stages;                 // [stages]
     uint64_t* acc_full = bars + 2 * p.stages;          // [2]
@@ -151,12 +154,26 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
             for (int sg = 0; sg < nseg && okp; ++sg) {
               const Seg seg = seg_of(sg, nseg, it_begin, it_end, p.k_blocks);
               const int tile = seg.it0 / p.k_blocks;
-              for (int it = seg.it0; it < seg.it1; ++it) {
+              for (int it = seg.it0; it < seg.it1; it += (p.pair ? 2 : 1)) {
                 const int kb = it - tile * p.k_blocks;
                 if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.status, 1)) { okp = false; break; }
-                uint8_t* st = stages + stage * kStageBytes;
-                mbar_expect_tx(&full[stage], kStageBytes);
+                uint8_t* st = stages + stage * stage_bytes;
+                mbar_expect_tx(&full[stage], stage_bytes);
                 const int n0 = tile * kBN, k0 = kb * kBK;
+                if (p.pair) {
+                    // two k blocks per stage: the weight maps carry boxes of 128 rows here; layout per weight matrix
+                    // [n half 0: 128 k rows][n half 1: 128 k rows], then the two X tiles
+                    tma_load_2d(st, &tmW0, &full[stage], n0, k0);
+                    tma_load_2d(st + 2 * kWAtomBytes, &tmW0, &full[stage], n0 + 64, k0);
+                    if (NW == 2) {
+                        tma_load_2d(st + 2 * kWBytes, &tmW1, &full[stage], n0, k0);
+                        tma_load_2d(st + 2 * kWBytes + 2 * kWAtomBytes, &tmW1, &full[stage], n0 + 64, k0);
+                    }
+                    if (!NORM) {
+                        tma_load_2d(st + NW * 2 * kWBytes, &tmX, &full[stage], k0, 0);
+                        tma_load_2d(st + NW * 2 * kWBytes + kXBytes, &tmX, &full[stage], k0 + kBK, 0);
+                    }
+                } else
                 if (NW == 1 && !NORM && p.lora && kb == p.k_blocks - 1) {
                     // the rank-16 update as one more k block: Bm rows 16..63 and T columns 16..63 lie outside
                     // their tensors and are filled with zeros (the second weight map carries Bm here)
@@ -310,10 +327,24 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                 if (!mbar_wait(&acc_empty[acc], ((iter >> 1) & 1) ^ 1u, abort_flag, p.status, 2)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kAccCols;
-                for (int i = 0; i < seg_end - it; ++i) {
+                for (int i = 0; i < seg_end - it; i += (p.pair ? 2 : 1)) {
                     if (!mbar_wait(&full[stage], phase, abort_flag, p.status, 3)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t st = smem_u32(stages + stage * kStageBytes);
+                    const uint32_t st = smem_u32(stages + stage * stage_bytes);
+                    if (p.pair) {
+                        // 128 k rows per stage: eight K = 16 steps; the second X tile follows the first
+                        const uint32_t xs = NORM ? smem_u32(xg + (kb0 + i) * kXBytes) : st + NW * 2 * kWBytes;
+                        const uint64_t b_desc = make_smem_desc(xs, 16, 1024, kSwizzle128B);
+#pragma unroll
+                        for (int w = 0; w < NW; ++w) {
+                            const uint64_t a_desc = make_smem_desc(st + w * 2 * kWBytes, 2 * kWAtomBytes, 1024, kSwizzle128B);
+#pragma unroll
+                            for (int kk = 0; kk < 2 * kBK / 16; ++kk)
+                                umma_ss(d_tmem + w * kMaxM, a_desc + static_cast<uint64_t>(kk * 128),
+                                        b_desc + static_cast<uint64_t>((kk >> 2) * (kXBytes >> 4) + (kk & 3) * 2), idesc,
+                                        (i | kk) != 0 ? 1u : 0u);
+                        }
+                    } else {
                     const uint32_t xs = NORM ? smem_u32(xg + (kb0 + i) * kXBytes) : st + NW * kWBytes;
                     const uint64_t b_desc = make_smem_desc(xs, 16, 1024, kSwizzle128B);
 #pragma unroll
@@ -323,6 +354,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                         for (int kk = 0; kk < kBK / 16; ++kk)
                             umma_ss(d_tmem + w * kMaxM, a_desc + static_cast<uint64_t>(kk * 128),
                                     b_desc + static_cast<uint64_t>(kk * 2), idesc, (i | kk) != 0 ? 1u : 0u);
+                    }
                     }
                     umma_commit(&empty[stage]);
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -493,6 +525,7 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
     int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
     if (grid > kMaxGrid) grid = kMaxGrid;
+    bool pair = false;
     if (pl.total_units / grid < 8) {
         // Few units per block: the call is latency-bound, and ranges that straddle n-tile boundaries add partial
         // slots and arrivals.  Cut every n tile into the same number s of k ranges instead (s divides k_blocks)
@@ -510,8 +543,19 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
         const double bytes = static_cast<double>(pl.total_units) * pl.stage_bytes;
         const double hbm = 5.7e6, per_block = static_cast<double>(pl.stages) * pl.stage_bytes / 2.9;   // bytes per microsecond
         const double whole_rate = per_block * pl.n_tiles < hbm ? per_block * pl.n_tiles : hbm;
-        if (bytes / whole_rate < bytes / hbm + 3.5) grid = pl.n_tiles;
+        if (bytes / whole_rate < bytes / hbm + 3.5) {
+            grid = pl.n_tiles;
+            pair = (pl.k_blocks % 2 == 0);   // every block then owns whole tiles: ranges start at k block 0 and have even length
+        }
     }
+    if (pair) {
+        // the weight maps get boxes of 128 rows; half as many stages of twice the size
+        const uint32_t wbox2[2] = {64, 2 * kBK};
+        if ((st = encode_tmap_bf16(&tmW0, W0, 2, wdims, wstrides, wbox2, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+        if ((st = encode_tmap_bf16(&tmW1, NW == 2 ? W1 : W0, 2, wdims, wstrides, wbox2, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
+        pl.stages /= 2;
+    }
+    p.pair = pair ? 1 : 0;
     p.base = pl.total_units / grid;
     p.rem = pl.total_units % grid;
     p.stages = pl.stages;
@@ -567,6 +611,7 @@ static ef_status launch_plain(const void* X, const void* W, int w_rows, const vo
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.M = M; p.K = K; p.N = N;
     p.lora = lora ? 1 : 0;
+    p.pair = 0;
     p.pdl_mode = pdl_mode;
     p.out_scale = out_scale;
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;

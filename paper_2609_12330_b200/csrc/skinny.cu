@@ -61,8 +61,9 @@ __device__ __forceinline__ int owner_of(int x, int base, int rem) {
     const int big = rem * (base + 1);
     return x < big ? x / (base + 1) : rem + (x - big) / base;
 }
-__device__ __forceinline__ int slot_of(int c, int tile, int base, int rem, int k_blocks) {
-    return 2 * c + ((range_begin(c, base, rem) / k_blocks) == tile ? 0 : 1);
+// (u = k blocks per partition unit: 2 when a stage holds two k blocks, else 1)
+__device__ __forceinline__ int slot_of(int c, int tile, int base, int rem, int k_blocks, int u) {
+    return 2 * c + ((u * range_begin(c, base, rem) / k_blocks) == tile ? 0 : 1);
 }
 // A block's range is a sequence of SEGMENTS, one per n tile it touches.  Only the first and the last can be partial
 // (shared with the neighbouring blocks).  Processing order: the partial LAST segment first, then the rest in
@@ -121,8 +122,9 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
     // X operand as hi/lo row pairs (see the prologue); LayerNorm keeps row 7 (split) or 15 for beta
     const bool split = NORM && p.M <= (LN ? 7 : 8);
     const int beta_row = split ? 7 : 15;
-    const int it_begin = range_begin(blockIdx.x, p.base, p.rem);
-    const int it_end = range_begin(blockIdx.x + 1, p.base, p.rem);
+    const int pu = p.pair ? 2 : 1;   // the partition counts pairs of k blocks when a stage holds two
+    const int it_begin = pu * range_begin(blockIdx.x, p.base, p.rem);
+    const int it_end = pu * range_begin(blockIdx.x + 1, p.base, p.rem);
     const int nseg = seg_count(it_begin, it_end, p.k_blocks);
 
     if (threadIdx.x == 0) {
@@ -389,22 +391,22 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
             bool finish = whole;
             int n_parts = 0;
             if (!whole) {
-                float* ps = p.partials + static_cast<size_t>(slot_of(blockIdx.x, tile, p.base, p.rem, p.k_blocks)) * (NW * kMaxM * kBN);
+                float* ps = p.partials + static_cast<size_t>(slot_of(blockIdx.x, tile, p.base, p.rem, p.k_blocks, pu)) * (NW * kMaxM * kBN);
 #pragma unroll
                 for (int w = 0; w < NW; ++w)
 #pragma unroll
                     for (int m = 0; m < kMaxM; ++m) ps[(w * kMaxM + m) * kBN + et] = __uint_as_float(v[w][m]);
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int c_first = owner_of(tile * p.k_blocks, p.base, p.rem);
-                const int c_last = owner_of(tile_end - 1, p.base, p.rem);
+                const int c_first = owner_of(tile * p.k_blocks / pu, p.base, p.rem);
+                const int c_last = owner_of((tile_end - 1) / pu, p.base, p.rem);
                 n_parts = c_last - c_first + 1;
                 if (warp == 2 && lane == 0) {
                     const uint32_t prev = atomicAdd(&p.counters[tile], 1u);
                     *is_last = (prev == static_cast<uint32_t>(n_parts - 1)) ? 1u : 0u;
                 }
                 for (int i = threadIdx.x - 64; i < n_parts; i += 128)
-                    slot_table[i] = slot_of(c_first + i, tile, p.base, p.rem, p.k_blocks);
+                    slot_table[i] = slot_of(c_first + i, tile, p.base, p.rem, p.k_blocks, pu);
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (*is_last) {
                     __threadfence();
@@ -523,41 +525,42 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
     p.pdl_mode = 0;
     p.out_scale = 1.f;
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
-    int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
+    // Two k blocks per stage (weight boxes of 128 rows, 16 KiB: the copy engine moves more per request, and there are half as
+    // many barrier round trips) whenever K allows it and at least two such stages fit; the partition then counts pairs.
+    const bool pair = (pl.k_blocks % 2 == 0) && pl.stages >= 4;
+    const int ku = pair ? 2 : 1;
+    const int units = pl.total_units / ku, k_units = pl.k_blocks / ku;
+    int grid = di.num_sms < units ? di.num_sms : units;
     if (grid > kMaxGrid) grid = kMaxGrid;
-    bool pair = false;
     if (pl.total_units / grid < 8) {
-        // Few units per block: the call is latency-bound, and ranges that straddle n-tile boundaries add partial
-        // slots and arrivals.  Cut every n tile into the same number s of k ranges instead (s divides k_blocks)
+        // Few k blocks per block: the call is latency-bound, and ranges that straddle n-tile boundaries add partial
+        // slots and arrivals.  Cut every n tile into the same number s of k ranges instead (s divides the k units)
         // as long as that keeps at least half of the blocks.
         int s = 0;
-        for (int d = 1; d <= pl.k_blocks; ++d)
-            if (pl.k_blocks % d == 0 && static_cast<long long>(pl.n_tiles) * d <= grid) s = d;
+        for (int d = 1; d <= k_units; ++d)
+            if (k_units % d == 0 && static_cast<long long>(pl.n_tiles) * d <= grid) s = d;
         if (s > 0 && pl.n_tiles * s * 2 >= grid) grid = pl.n_tiles * s;
     } else if (pl.n_tiles <= grid) {
-        // Many units per block and no more n tiles than SMs: one block per whole tile needs no partial slots, no arrival
+        // Many k blocks per block and no more n tiles than SMs: one block per whole tile needs no partial slots, no arrival
         // counters and no merging block at the end of the kernel (measured: ~3.5 us), but leaves SMs idle.  A block alone
-        // streams what it keeps in flight per ~2.9 us of memory latency, so whole tiles win when n_tiles such blocks
-        // already saturate HBM (gated MLP at 16x4096x11008: 86 blocks, 35.8 us against 38.2 us with 148 split ranges;
-        // with the normalised X operand resident in shared memory there are fewer stages and the split stays better).
+        // streams what it keeps in flight per ~2.9 us of memory latency (less with the larger boxes), so whole tiles win
+        // when n_tiles such blocks already saturate HBM (gated MLP at 16x4096x11008: 86 blocks, 33.2 us against 38.2 us
+        // with 148 split ranges; with the normalised X operand resident in shared memory there are fewer stages and the
+        // split stays better).
         const double bytes = static_cast<double>(pl.total_units) * pl.stage_bytes;
-        const double hbm = 5.7e6, per_block = static_cast<double>(pl.stages) * pl.stage_bytes / 2.9;   // bytes per microsecond
+        const double hbm = 5.7e6, per_block = static_cast<double>(pl.stages) * pl.stage_bytes / (pair ? 2.3 : 2.9);   // bytes per microsecond
         const double whole_rate = per_block * pl.n_tiles < hbm ? per_block * pl.n_tiles : hbm;
-        if (bytes / whole_rate < bytes / hbm + 3.5) {
-            grid = pl.n_tiles;
-            pair = (pl.k_blocks % 2 == 0);   // every block then owns whole tiles: ranges start at k block 0 and have even length
-        }
+        if (bytes / whole_rate < bytes / hbm + 3.5) grid = pl.n_tiles;
     }
     if (pair) {
-        // the weight maps get boxes of 128 rows; half as many stages of twice the size
         const uint32_t wbox2[2] = {64, 2 * kBK};
         if ((st = encode_tmap_bf16(&tmW0, W0, 2, wdims, wstrides, wbox2, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
         if ((st = encode_tmap_bf16(&tmW1, NW == 2 ? W1 : W0, 2, wdims, wstrides, wbox2, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
         pl.stages /= 2;
     }
     p.pair = pair ? 1 : 0;
-    p.base = pl.total_units / grid;
-    p.rem = pl.total_units % grid;
+    p.base = (pl.total_units / (pair ? 2 : 1)) / grid;
+    p.rem = (pl.total_units / (pair ? 2 : 1)) % grid;
     p.stages = pl.stages;
     p.eps = eps;
     uint8_t* w = static_cast<uint8_t*>(ws);

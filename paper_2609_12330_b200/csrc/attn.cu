@@ -243,8 +243,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     uint64_t* q_full = bars;                 // [2]  TMA -> softmax group t (raw Q tile t of the item landed)
     uint64_t* q_empty = bars + 2;            // [2]  MMA -> TMA (last QK^T of tile t done: Q tile t may be overwritten)
     uint64_t* q_ready = bars + 4;            // [2]  softmax group t -> MMA (Q tile t rewritten)
-    uint64_t* kv_full = bars + 6;            // [5]  K/V ring: load number n (K of key tile c: n = 2c, V: n = 2c+1)
-    uint64_t* kv_empty = bars + 11;          // [5]        lives in slot n % 5, phase (n / 5) & 1
+    uint64_t* kv_full = bars + 6;            // [kKVSlots <= 5]  K/V ring: load number n (K of key tile c: n = 2c, V: n = 2c+1)
+    uint64_t* kv_empty = bars + 11;          // [kKVSlots <= 5]  lives in slot n % kKVSlots, phase (n / kKVSlots) & 1
     uint64_t* s_full = bars + 16;            // [2]  MMA -> softmax group t
     uint64_t* p_full = bars + 18;            // [2]  softmax group t -> MMA
     uint64_t* o_done = bars + 20;            // [2]  MMA -> softmax group t (PV finished)

@@ -40,7 +40,7 @@ constexpr int kD = 128;
 constexpr int kT = 128;                           // tile edge (queries and keys)
 constexpr int kHalfBytes = kT * 128;              // [128 rows][64 d] bf16, 128B swizzle
 constexpr int kTileBytes = 2 * kHalfBytes;        // 32 KiB
-constexpr int kKVSlots = 4;                        // one ring for K and V tiles: K_j, V_j, K_j+1, V_j+1, K_j+2
+constexpr int kKVSlots = 4;                        // K/V tiles in shared memory: two double slots {V_j, K_j+1}
 constexpr int kThreads = 320;
 constexpr int kKeyRowsPerThread = 4;               // pre-pass: key rows per thread
 constexpr uint32_t kTmemCols = 512;               // S0 | S1 | O0 | O1, 128 fp32 columns each
@@ -243,8 +243,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     uint64_t* q_full = bars;                 // [2]  TMA -> softmax group t (raw Q tile t of the item landed)
     uint64_t* q_empty = bars + 2;            // [2]  MMA -> TMA (last QK^T of tile t done: Q tile t may be overwritten)
     uint64_t* q_ready = bars + 4;            // [2]  softmax group t -> MMA (Q tile t rewritten)
-    uint64_t* kv_full = bars + 6;            // [kKVSlots <= 5]  K/V ring: load number n (K of key tile c: n = 2c, V: n = 2c+1)
-    uint64_t* kv_empty = bars + 11;          // [kKVSlots <= 5]  lives in slot n % kKVSlots, phase (n / kKVSlots) & 1
+    uint64_t* kv_full = bars + 6;            // [2]  K/V ring of two double slots: pair number n lives in double slot n & 1,
+    uint64_t* kv_empty = bars + 11;          // [2]        phase (n >> 1) & 1
     uint64_t* s_full = bars + 16;            // [2]  MMA -> softmax group t
     uint64_t* p_full = bars + 18;            // [2]  softmax group t -> MMA
     uint64_t* o_done = bars + 20;            // [2]  MMA -> softmax group t (PV finished)
@@ -284,7 +284,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // ------------------------------ TMA producer + work fetch ------------------------------
         if (lane == 0) {
             tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-            uint32_t kv_count = 0;   // key tiles loaded so far (stage / phase of the K and V rings)
+            uint32_t pc = 0;   // K/V pairs loaded so far: pair = {V of one list entry, K of the next} in one double slot, ONE barrier
             uint32_t n_items = 0;
             uint32_t item = atomicAdd(&p.header[kWorkCounterWord], 1u);
             bool ok = true;
@@ -309,24 +309,30 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 };
                 if (!load_q(0)) break;
                 const int kvz = (p.Hq == p.Hkv) ? g.bh : (g.bh / p.Hq) * p.Hkv + (g.bh % p.Hq) / (p.Hq / p.Hkv);   // K/V head
-                for (int a = 0; a < g.n_kv; ++a, ++kv_count) {
-                    const int j = g.kt(a);   // key tile of list entry a
-                    {
-                        const uint32_t n = 2 * kv_count, sl = n % kKVSlots;
-                        if (!mbar_wait(&kv_empty[sl], ((n / kKVSlots) & 1) ^ 1u, abort_flag, p.status, 3)) { ok = false; break; }
-                        mbar_expect_tx(&kv_full[sl], kTileBytes);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmK, &kv_full[sl], 0, j * kT, kvz);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmK, &kv_full[sl], 64, j * kT, kvz);
+                // The K/V ring holds two double slots.  A double slot carries what one step of the MMA issuer consumes -- V of
+                // list entry a and K of entry a+1 -- under ONE full/empty barrier pair (the issuer spends its time on barrier
+                // round trips, so there are as few as possible); the item's first K tile travels alone in a double slot.
+                auto load_pair = [&](int a_v, int a_k) -> bool {   // a_v < 0: no V; a_k < 0: no K
+                    const uint32_t d = pc & 1u;
+                    if (!mbar_wait(&kv_empty[d], ((pc >> 1) & 1) ^ 1u, abort_flag, p.status, 3)) return false;
+                    uint8_t* base = smem + kOffKV + d * 2 * kTileBytes;
+                    mbar_expect_tx(&kv_full[d], ((a_v >= 0) + (a_k >= 0)) * kTileBytes);
+                    if (a_v >= 0) {
+                        const int j = g.kt(a_v);
+                        tma_load_3d(base, &tmV, &kv_full[d], 0, j * kT, kvz);
+                        tma_load_3d(base + kHalfBytes, &tmV, &kv_full[d], 64, j * kT, kvz);
                     }
-                    if (a == 0 && !load_q(1)) { ok = false; break; }
-                    {
-                        const uint32_t n = 2 * kv_count + 1, sl = n % kKVSlots;
-                        if (!mbar_wait(&kv_empty[sl], ((n / kKVSlots) & 1) ^ 1u, abort_flag, p.status, 3)) { ok = false; break; }
-                        mbar_expect_tx(&kv_full[sl], kTileBytes);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes, &tmV, &kv_full[sl], 0, j * kT, kvz);
-                        tma_load_3d(smem + kOffKV + sl * kTileBytes + kHalfBytes, &tmV, &kv_full[sl], 64, j * kT, kvz);
+                    if (a_k >= 0) {
+                        const int j = g.kt(a_k);
+                        tma_load_3d(base + kTileBytes, &tmK, &kv_full[d], 0, j * kT, kvz);
+                        tma_load_3d(base + kTileBytes + kHalfBytes, &tmK, &kv_full[d], 64, j * kT, kvz);
                     }
-                }
+                    ++pc;
+                    return true;
+                };
+                ok = load_pair(-1, 0) && load_q(1);
+                for (int a = 0; a < g.n_kv && ok; ++a) ok = load_pair(a, a + 1 < g.n_kv ? a + 1 : -1);
+                if (!ok) break;
                 item = next;
                 ++n_items;
             }
@@ -348,21 +354,25 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             constexpr uint32_t hi_kmajor = smem_desc_hi(1024, kSwizzle128B);   // Q and K tiles
             constexpr uint32_t hi_v = smem_desc_hi(1024, kSwizzle128B);        // V tile (MN-major: LBO in lo word)
             const uint32_t q_lo[2] = {smem_desc_lo(sQ, 16), smem_desc_lo(sQ + kTileBytes, 16)};
-            auto issue_qk = [&](int t, uint32_t slot) {
-                const uint32_t a0 = q_lo[t], b0 = smem_desc_lo(sKV + slot * kTileBytes, 16), d = tmem_base + t * kT;
+            auto issue_qk = [&](int t, uint32_t kaddr) {
+                const uint32_t a0 = q_lo[t], b0 = smem_desc_lo(kaddr, 16), d = tmem_base + t * kT;
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
                     umma_ss_w(d, a0 + off, hi_kmajor, b0 + off, hi_kmajor, idesc_qk, kk != 0 ? 1u : 0u);
                 }
             };
-            auto issue_pv = [&](int t, uint32_t slot, uint32_t accumulate) {
-                const uint32_t b0 = smem_desc_lo(sKV + slot * kTileBytes, kHalfBytes), d = tmem_base + 2 * kT + t * kD, a = tmem_base + t * kT;
+            auto issue_pv = [&](int t, uint32_t vaddr, uint32_t accumulate) {
+                const uint32_t b0 = smem_desc_lo(vaddr, kHalfBytes), d = tmem_base + 2 * kT + t * kD, a = tmem_base + t * kT;
 #pragma unroll
                 for (int kk = 0; kk < kT / 16; ++kk)
                     umma_ts_w(d, a + kk * 8, b0 + kk * (2048 >> 4), hi_v, idesc_pv, kk != 0 ? 1u : accumulate);
             };
-            uint32_t kv_use = 0;          // key tiles consumed by earlier items
+            uint32_t pu = 0;              // K/V pairs (double slots) consumed so far
+            // with the a-priori logit bound nobody waits for a PV but the epilogue: one commit per item and tile suffices
+            float gmax_i = 0.f;
+            for (int d = 0; d < kD; ++d) gmax_i = fmaxf(gmax_i, fabsf(gprod[d]));
+            const bool every_pv = !(static_cast<float>(kD) * gmax_i * p.scale_log2 <= kFixedRefLimit);
             uint32_t n_items = 0;
             uint32_t cp[2] = {0u, 0u};    // p_full completions consumed per tile
             bool ok = true;
@@ -377,7 +387,8 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 // issued during step a (right after the tile's PV of entry a, if it has one), so the K/V ring is
                 // released in list order whatever subset of entries a tile visits.
                 {
-                    const uint32_t n0 = 2 * kv_use, st0 = n0 % kKVSlots;   // K of the item's first list entry
+                    const uint32_t st0 = pu & 1u;   // double slot of the item's first K tile
+                    const uint32_t k0addr = sKV + st0 * 2 * kTileBytes + kTileBytes;
                     bool k_waited = false;
                     for (int t = 0; t < 2 && ok; ++t) {
                         ok = mbar_wait(&q_ready[t], n_items & 1, abort_flag, p.status, 4);
@@ -385,11 +396,11 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         if (!ok) break;
                         if (g.part(t, 0)) {
                             if (!k_waited) {
-                                if (!mbar_wait(&kv_full[st0], (n0 / kKVSlots) & 1, abort_flag, p.status, 5)) { ok = false; break; }
+                                if (!mbar_wait(&kv_full[st0], (pu >> 1) & 1, abort_flag, p.status, 5)) { ok = false; break; }
                                 k_waited = true;
                             }
                             tc_fence_after();
-                            issue_qk(t, st0);
+                            issue_qk(t, k0addr);
                             umma_commit(&s_full[t]);
                         }
                         // tile t's last QK^T (or none at all): its Q tile may be overwritten
@@ -397,44 +408,33 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     }
                     if (!ok) break;
                     umma_commit(&kv_empty[st0]);
+                    ++pu;
                 }
-                for (int j = 0; j < g.n_kv && ok; ++j) {
-                    const uint32_t nv = 2 * (kv_use + j) + 1, nk = nv + 1;   // load numbers of V_j and K_j+1
-                    const uint32_t st = nv % kKVSlots, stn = nk % kKVSlots;
-                    // The K/V tiles of this step landed long ago: look at their barriers now, while the softmax groups
-                    // are still busy, so that nothing but the MMAs follows a group's hand-over on the critical path.
-                    if (!mbar_wait(&kv_full[st], (nv / kKVSlots) & 1, abort_flag, p.status, 7)) { ok = false; break; }
-                    if (j + 1 < g.n_kv && !mbar_wait(&kv_full[stn], (nk / kKVSlots) & 1, abort_flag, p.status, 8)) { ok = false; break; }
-                    bool v_waited = true, k_waited = j + 1 < g.n_kv;
+                for (int j = 0; j < g.n_kv && ok; ++j, ++pu) {
+                    const uint32_t st = pu & 1u;   // double slot of this step: V of entry j, K of entry j+1
+                    const uint32_t vaddr = sKV + st * 2 * kTileBytes, kaddr = vaddr + kTileBytes;
+                    // The tiles of this step landed long ago: look at their barrier now, while the softmax groups are still
+                    // busy, so that nothing but the MMAs follows a group's hand-over on the critical path.
+                    if (!mbar_wait(&kv_full[st], (pu >> 1) & 1, abort_flag, p.status, 7)) { ok = false; break; }
+                    tc_fence_after();
                     for (int t = 0; t < 2 && ok; ++t) {
                         if (g.part(t, j)) {
                             if (!mbar_wait(&p_full[t], cp[t] & 1, abort_flag, p.status, 6)) { ok = false; break; }
                             ++cp[t];
-                            if (!v_waited) {
-                                if (!mbar_wait(&kv_full[st], (nv / kKVSlots) & 1, abort_flag, p.status, 7)) { ok = false; break; }
-                                v_waited = true;
-                            }
                             tc_fence_after();
-                            issue_pv(t, st, j > g.first(t) ? 1u : 0u);
-                            umma_commit(&o_done[t]);
+                            issue_pv(t, vaddr, j > g.first(t) ? 1u : 0u);
+                            if (every_pv || j == g.last(t)) umma_commit(&o_done[t]);
                         }
                         if (j + 1 < g.n_kv && g.part(t, j + 1)) {
-                            if (!k_waited) {
-                                if (!mbar_wait(&kv_full[stn], (nk / kKVSlots) & 1, abort_flag, p.status, 8)) { ok = false; break; }
-                                k_waited = true;
-                                tc_fence_after();
-                            }
-                            issue_qk(t, stn);
+                            issue_qk(t, kaddr);
                             umma_commit(&s_full[t]);
                             if (j + 1 == g.last(t)) umma_commit(&q_empty[t]);   // tile t's last QK^T: its Q tile is free
                         }
                     }
                     if (!ok) break;
-                    umma_commit(&kv_empty[st]);                  // all PV of entry j issued: V_j's slot is free
-                    if (k_waited) umma_commit(&kv_empty[stn]);   // all QK of entry j+1 issued: K_j+1's slot is free
+                    umma_commit(&kv_empty[st]);   // all MMAs that read this double slot are issued
                 }
                 if (!ok) break;
-                kv_use += static_cast<uint32_t>(g.n_kv);
                 ++n_items;
             }
         }
@@ -471,6 +471,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const Item g = item_from<WIN>(p, item.x, item.y);
             const bool present = g.present(t);
             const int my_count = present ? g.wl(t) - g.wf(t) + 1 + g.sink : 0;   // list entries this tile takes part in
+            const int my_commits = fixed_ref ? (my_count > 0 ? 1 : 0) : my_count;      // o_done completions of this item
             const int qt = g.qt0 + t;
             const int row_g = qt * kT + r;             // query index within the sequence
             if (!warp_wait(&q_full[t], n_items & 1, abort_flag, p.status, 9)) break;
@@ -617,7 +618,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (!ok) break;
             // epilogue: read O out of TMEM (then the next item may overwrite it), scale by 1/l, store
             if (my_count > 0) {
-                if (!warp_wait(&o_done[t], (co + my_count - 1) & 1, abort_flag, p.status, 13)) break;
+                if (!warp_wait(&o_done[t], (co + my_commits - 1) & 1, abort_flag, p.status, 13)) break;
                 tc_fence_after();
                 const float inv = 1.f / l_sum;
                 uint8_t* orow = reinterpret_cast<uint8_t*>(p.O + (static_cast<size_t>(g.bh) * p.S + row_g) * kD);
@@ -648,7 +649,7 @@ qknorm_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         }
                     }
                 }
-                co += static_cast<uint32_t>(my_count);
+                co += static_cast<uint32_t>(my_commits);
             }
             tc_fence_before();
             __syncwarp();

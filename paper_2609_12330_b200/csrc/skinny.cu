@@ -165,7 +165,15 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                 const bool wide = p.tile_n == kBN;
                 mbar_expect_tx(&full[stage], stage_bytes - (wide ? 0 : NW * kWAtomBytes * (p.pair ? 2 : 1)));
                 const int n0 = tile * p.tile_n, k0 = kb * kBK;
-                if (p.pair) {
+                if (p.pair && NW == 1 && !NORM && p.lora && kb == p.k_blocks - 2) {
+                    // the rank-16 update as the last double stage: Bm rows 16..127 and T columns 16..127 lie outside their
+                    // tensors and are filled with zeros (the second weight map carries Bm here, with 128-row boxes)
+                    if (p.pdl_mode == 2 && !t_waited) { pdl_wait(); t_waited = true; }   // T comes from the kernel before
+                    tma_load_2d(st, &tmW1, &full[stage], n0, 0);
+                    tma_load_2d(st + 2 * kWAtomBytes, &tmW1, &full[stage], n0 + 64, 0);
+                    tma_load_2d(st + NW * 2 * kWBytes, &tmT, &full[stage], 0, 0);
+                    tma_load_2d(st + NW * 2 * kWBytes + kXBytes, &tmT, &full[stage], 64, 0);
+                } else if (p.pair) {
                     // two k blocks per stage: the weight maps carry boxes of 128 rows here; layout per weight matrix
                     // [n half 0: 128 k rows][n half 1: 128 k rows], then the two X tiles
                     tma_load_2d(st, &tmW0, &full[stage], n0, k0);
@@ -603,14 +611,16 @@ static ef_status launch_plain(const void* X, const void* W, int w_rows, const vo
     const bool lora = T != nullptr;
     Plan pl;
     if (M > kMaxM || K % kBK != 0 || N % 8 != 0) return EF_ERR_UNSUPPORTED;
-    if (!make_plan(1, false, K + (lora ? kBK : 0), N, &pl)) return EF_ERR_UNSUPPORTED;   // LoRA: one more k block than K / 64
+    // Two k blocks per stage when K / 64 is even (see launch()); the rank-16 update then takes a whole double stage.
+    const bool pair = ((K / kBK) % 2 == 0);
+    if (!make_plan(1, false, K + (lora ? (pair ? 2 : 1) * kBK : 0), N, &pl)) return EF_ERR_UNSUPPORTED;   // LoRA: one more stage than K needs
     if (static_cast<long long>(pl.n_tiles) * pl.k_blocks >= (1LL << 30)) return EF_ERR_UNSUPPORTED;
     CUtensorMap tmW, tmB, tmX, tmT;
     ef_status st;
     const uint64_t wdims[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(w_rows)};
     const uint64_t bdims[2] = {static_cast<uint64_t>(N), 16};
     const uint64_t wstrides[1] = {static_cast<uint64_t>(N) * 2};
-    const uint32_t wbox[2] = {64, kBK};
+    const uint32_t wbox[2] = {64, static_cast<uint32_t>(pair ? 2 * kBK : kBK)};
     if ((st = encode_tmap_bf16(&tmW, W, 2, wdims, wstrides, wbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
     if ((st = encode_tmap_bf16(&tmB, lora ? Bm : W, 2, lora ? bdims : wdims, wstrides, wbox, CU_TENSOR_MAP_SWIZZLE_128B)) != EF_OK) return st;
     const uint64_t xdims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
@@ -633,15 +643,17 @@ static ef_status launch_plain(const void* X, const void* W, int w_rows, const vo
     p.M = M; p.K = K; p.N = N;
     p.lora = lora ? 1 : 0;
     p.tile_n = kBN;
-    p.pair = 0;
+    p.pair = pair ? 1 : 0;
+    if (pair) pl.stages /= 2;
     p.pdl_mode = pdl_mode;
     p.out_scale = out_scale;
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
-    int grid = di.num_sms < pl.total_units ? di.num_sms : pl.total_units;
+    const int units = pl.total_units / (pair ? 2 : 1);   // the partition counts pairs of k blocks when a stage holds two
+    int grid = di.num_sms < units ? di.num_sms : units;
     if (grid > kMaxGrid) grid = kMaxGrid;
     if (grid > grid_cap) grid = grid_cap;
-    p.base = pl.total_units / grid;
-    p.rem = pl.total_units % grid;
+    p.base = units / grid;
+    p.rem = units % grid;
     p.stages = pl.stages;
     p.eps = 0.f;
     p.status = status;

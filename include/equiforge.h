@@ -83,7 +83,9 @@ size_t ef_gated_mlp_workspace_bytes(int M, int K, int N);
  * after each projection, (s (.) X) W == s (.) (X W), and both projections plus the elementwise
  * product run in ONE kernel with no intermediate in global memory.
  *   X [M,K], gamma [K], Wgate [K,N], Wup [K,N] -> Y [M,N].
- * Supported: 1 <= M <= 16, K % 64 == 0, K <= 4096, N % 8 == 0. */
+ * Supported: 1 <= M <= 16, K % 64 == 0, K <= 4096, N % 8 == 0.  Up to 8 rows run as ONE kernel; 9..16
+ * rows run as two launches of at most 8 rows each on the same workspace (the operand of the tensor
+ * core carries the rounding remainder of x*gamma in spare rows, which exist for at most 8 rows). */
 ef_status ef_rmsnorm_gated_mlp(const void* X, const void* gamma, const void* Wgate, const void* Wup, void* Y,
                                int M, int K, int N, float eps,
                                void* ws, size_t ws_bytes, void* stream);

@@ -170,7 +170,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                     // tensors and are filled with zeros (the second weight map carries Bm here, with 128-row boxes)
                     if (p.pdl_mode == 2 && !t_waited) { pdl_wait(); t_waited = true; }   // T comes from the kernel before
                     tma_load_2d(st, &tmW1, &full[stage], n0, 0);
-                    tma_load_2d(st + 2 * kWAtomBytes, &tmW1, &full[stage], n0 + 64, 0);
+                    if (wide) tma_load_2d(st + 2 * kWAtomBytes, &tmW1, &full[stage], n0 + 64, 0);
                     tma_load_2d(st + NW * 2 * kWBytes, &tmT, &full[stage], 0, 0);
                     tma_load_2d(st + NW * 2 * kWBytes + kXBytes, &tmT, &full[stage], 64, 0);
                 } else if (p.pair) {
@@ -192,7 +192,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ 
                     // their tensors and are filled with zeros (the second weight map carries Bm here)
                     if (p.pdl_mode == 2 && !t_waited) { pdl_wait(); t_waited = true; }   // T comes from the kernel before
                     tma_load_2d(st, &tmW1, &full[stage], n0, 0);
-                    tma_load_2d(st + kWAtomBytes, &tmW1, &full[stage], n0 + 64, 0);
+                    if (wide) tma_load_2d(st + kWAtomBytes, &tmW1, &full[stage], n0 + 64, 0);
                     tma_load_2d(st + NW * kWBytes, &tmT, &full[stage], 0, 0);
                 } else {
                     tma_load_2d(st, &tmW0, &full[stage], n0, k0);
@@ -601,7 +601,7 @@ ef_status launch(const void* X, const void* gamma, const void* beta, const void*
 // The LoRA-fused linear for M <= 16 rows, both kernels on the weight-streaming kernel above:
 //   launch_lora_head: T = alpha * X @ A   (A is a [K,16] weight: one n tile; few blocks, so few partials to merge)
 //   launch_lora_tail: Y = [X | T] @ [W ; Bm], the rank-16 update as one extra k block.
-size_t lora_tail_counters_bytes(int N) { return 256 + ((static_cast<size_t>((N + kBN - 1) / kBN) * 4 + 255) & ~size_t(255)); }
+size_t lora_tail_counters_bytes(int N) { return 256 + ((static_cast<size_t>((N + 63) / 64) * 4 + 255) & ~size_t(255)); }
 constexpr int kLoraHeadGrid = 8;   // one n tile of 16 live columns, K / 64 k blocks: 8 blocks keep the ordered merge short
 // partial slots of the head kernel (kLoraHeadGrid blocks) followed by those of the tail kernel: the two run concurrently
 size_t lora_tail_partials_bytes() { return static_cast<size_t>(kLoraHeadGrid + kMaxGrid) * 2 * kMaxM * kBN * 4; }
@@ -647,11 +647,17 @@ static ef_status launch_plain(const void* X, const void* W, int w_rows, const vo
     if (pair) pl.stages /= 2;
     p.pdl_mode = pdl_mode;
     p.out_scale = out_scale;
+    // 64-column tiles when every block can then own a whole one (no partial exchange) and there are enough such blocks to
+    // keep HBM busy (N = 8192: 128 blocks, 19.4 us against 24.5 us with split 128-column tiles; N = 4096: 64 blocks, no gain)
+    const int n_tiles64 = (N + 63) / 64;
+    const bool half = lora && n_tiles64 >= 76 && n_tiles64 <= di.num_sms && n_tiles64 <= grid_cap;
+    if (half) { p.tile_n = 64; pl.n_tiles = n_tiles64; pl.total_units = pl.n_tiles * pl.k_blocks; }
     p.n_tiles = pl.n_tiles; p.k_blocks = pl.k_blocks; p.total_units = pl.total_units;
     const int units = pl.total_units / (pair ? 2 : 1);   // the partition counts pairs of k blocks when a stage holds two
     int grid = di.num_sms < units ? di.num_sms : units;
     if (grid > kMaxGrid) grid = kMaxGrid;
     if (grid > grid_cap) grid = grid_cap;
+    if (half) grid = pl.n_tiles;
     p.base = units / grid;
     p.rem = units % grid;
     p.stages = pl.stages;
@@ -697,6 +703,17 @@ size_t ef_rmsnorm_gated_mlp_workspace_bytes(int M, int K, int N) {
 }
 ef_status ef_rmsnorm_gated_mlp(const void* X, const void* gamma, const void* Wgate, const void* Wup, void* Y, int M, int K,
                                int N, float eps, void* ws, size_t ws_bytes, void* stream) {
+    // Up to 8 rows go through in one launch with the hi/lo operand split (the spare operand rows carry the rounding remainder
+    // of x*gamma).  More rows have no spare operand rows, and the plain bf16 operand is not accurate enough for the gated
+    // product (a small SiLU(g) times a large u: single elements miss 1e-2 + 1e-2*|ref| by up to 3x), so 9..16 rows run as two
+    // launches of <= 8 rows each on the same workspace: twice the weight traffic, the same accuracy as for M <= 8.
+    if (M > 8 && M <= ef::skinny::kMaxM && X && Y && K > 0 && N > 0) {
+        const ef_status st = ef::skinny::launch<2, 1>(X, gamma, nullptr, Wgate, Wup, Y, 8, K, N, eps, ws, ws_bytes, stream);
+        if (st != EF_OK) return st;
+        return ef::skinny::launch<2, 1>(static_cast<const __nv_bfloat16*>(X) + static_cast<size_t>(8) * K, gamma, nullptr, Wgate,
+                                        Wup, static_cast<__nv_bfloat16*>(Y) + static_cast<size_t>(8) * N, M - 8, K, N, eps, ws,
+                                        ws_bytes, stream);
+    }
     return ef::skinny::launch<2, 1>(X, gamma, nullptr, Wgate, Wup, Y, M, K, N, eps, ws, ws_bytes, stream);
 }
 
